@@ -1,0 +1,447 @@
+"""Benchmark of the tree-verification hot path (one B200 per process).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2]
+
+A "step" is one verify step of the LLaVA-1.6-7B-shaped workload: L = 32 per-layer
+tree-verification attention launches over 32 distinct KV caches (prefix 3008, 60-node
+tree), one vocabulary argmax over 60 x 32000 fp32 logits, and one fused path-walk +
+KV-compaction launch. Inputs are seeded and synthetic. Rank 0 prints ONE JSON line.
+
+For N > 1 every rank runs an independent replica on its own GPU (the path has no
+exchange step); the whole-job value is the sum of steps over ranks divided by the
+slowest rank's time (weak scaling).
+
+`--impl reference` times the fp64 CPU oracle (test infrastructure) on the host cores.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "verify_steps_per_s"
+UNIT = "steps/s"
+N_INPUT_SETS = 4          # distinct (tree, logits) sets rotated over the steps
+
+
+# ----------------------------------------------------------------------------- inputs
+
+
+def make_step_inputs(cfg, n_sets):
+    """Host-side per-step inputs: trees, draft tokens, planted logits (fresh per set)."""
+    sets = []
+    for s in range(n_sets):
+        rng = np.random.default_rng([cfg.seed, s])
+        parents, drafts, logits = [], [], []
+        for b in range(cfg.B):
+            p = wl.eagle2_like_tree(rng, cfg.T, cfg.max_depth)
+            d = wl.sibling_distinct_tokens(rng, p, cfg.V)
+            lg, _ = wl.planted_logits(rng, p, d, cfg.V, plant_len=int(rng.integers(0, cfg.max_depth + 1)))
+            parents.append(p), drafts.append(d), logits.append(lg)
+        sets.append((np.array(parents, dtype=np.int32), np.array(drafts, dtype=np.int32), np.stack(logits)))
+    return sets
+
+
+# ----------------------------------------------------------------------------- clocks
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def sample(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+            names = {
+                "hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown,
+                "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown,
+                "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown,
+                "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap,
+                "hw_power_brake": nv.nvmlClocksEventReasonHwPowerBrakeSlowdown,
+            }
+            for k, bit in names.items():
+                if r & bit:
+                    self.reasons.add(k)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample()
+            self._stop.wait(0.005)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+
+
+def oracle_sample(cfg, layers_sampled, repeats=1):
+    """Times the CPU oracle on `layers_sampled` layers of one verify step (all sequences and
+    heads) plus the argmax / acceptance / compaction of that step; returns the estimated
+    seconds per full step and the pieces."""
+    import oracle
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    rng = np.random.default_rng([cfg.seed, 99])
+    P = wl.draw_prefix_lens(cfg, np.random.default_rng(cfg.seed))
+    S_cap = cfg.s_cap
+    Ls = layers_sampled
+    q = wl.normal_bf16_bits(rng, (Ls, cfg.B, cfg.H, cfg.T, cfg.D))
+    k = wl.normal_bf16_bits(rng, (Ls, cfg.B, cfg.H, S_cap, cfg.D))
+    v = wl.normal_bf16_bits(rng, (Ls, cfg.B, cfg.H, S_cap, cfg.D))
+    parents, drafts, logits = make_step_inputs(cfg, 1)[0]
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        masks = [oracle.tree_mask_bits(parents[b]) for b in range(cfg.B)]
+        for l in range(Ls):
+            for b in range(cfg.B):
+                for h in range(cfg.H):
+                    oracle.attention.tree_attn_bits(q[l, b, h], k[l, b, h], v[l, b, h], int(P[b]), masks[b])
+        t1 = time.perf_counter()
+        tok = oracle.vocab_argmax(logits)
+        idx = np.full((cfg.B, 64), -1, dtype=np.int32)
+        n = np.zeros(cfg.B, dtype=np.int32)
+        for b in range(cfg.B):
+            path, n[b], _ = oracle.accept_topdown(parents[b], drafts[b], tok[b])
+            idx[b, :len(path)] = path
+        t2 = time.perf_counter()
+        oracle.kv_compact(k, v, P, idx, n)
+        t3 = time.perf_counter()
+        est = (t1 - t0) * cfg.L / Ls + (t2 - t1) + (t3 - t2) * cfg.L / Ls
+        piece = {"attn_s_per_layer": (t1 - t0) / Ls, "argmax_accept_s": t2 - t1,
+                 "compact_s_per_layer": (t3 - t2) / Ls, "est_step_s": est, "measured_s": t3 - t0}
+        if best is None or est < best["est_step_s"]:
+            best = piece
+    return best, cores
+
+
+def run_reference(args, cfg):
+    """The oracle as the reference arm: each step is a bounded sample (a few layers)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    Ls = 2 if cfg.L >= 2 else 1
+    for _ in range(args.warmup):
+        oracle_sample(cfg, 1)
+    ests = []
+    t0 = time.perf_counter()
+    cores = 1
+    for _ in range(args.steps):
+        piece, cores = oracle_sample(cfg, Ls)
+        ests.append(piece["est_step_s"])
+    wall = time.perf_counter() - t0
+    est = float(np.mean(ests))
+    sample = (f"each step: oracle on {Ls} of {cfg.L} layers (all {cfg.B * cfg.H} sequence-heads) + full argmax/"
+              f"accept + compaction of those layers; attention and compaction time scaled by {cfg.L}/{Ls}")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": 1.0 / est, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg),
+        "cpu_baseline": {"value": 1.0 / est, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": 1.0 / est, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "wall_s": wall,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(cfg):
+    return {"workload": f"{cfg.name}: {cfg.note}", "L": cfg.L, "H": cfg.H, "D": cfg.D, "B": cfg.B, "T": cfg.T,
+            "prefix": cfg.prefix_nominal, "vocab": cfg.V,
+            "l2": "inputs larger than L2: every step streams L distinct KV caches "
+                  f"({cfg.L} x {2 * cfg.H * (cfg.prefix_nominal + cfg.T) * cfg.D * 2 / 1e6:.1f} MB)"}
+
+
+# ----------------------------------------------------------------------------- GPU arm
+
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2509_11815_b200 as sv
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    sv.load_library()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    L, B, H, T, D, V = cfg.L, cfg.B, cfg.H, cfg.T, cfg.D, cfg.V
+    S_cap = cfg.s_cap
+    P_host = wl.draw_prefix_lens(cfg, np.random.default_rng(cfg.seed))
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.seed + rank)
+    bf = dict(dtype=torch.bfloat16, device=dev)
+    k_cache = torch.randn((L, B, H, S_cap, D), generator=gen, **bf)
+    v_cache = torch.randn((L, B, H, S_cap, D), generator=gen, **bf)
+    q = torch.randn((L, B, H, T, D), generator=gen, **bf)
+    out = torch.empty_like(q)
+    i32 = dict(dtype=torch.int32, device=dev)
+    prefix_len = torch.tensor(P_host, **i32)
+    sets_host = make_step_inputs(cfg, N_INPUT_SETS)
+    sets = []
+    for parents, drafts, logits in sets_host:
+        par = torch.tensor(parents, **i32)
+        mask = torch.zeros((B, T), dtype=torch.int64, device=dev)
+        sv.specvlm_tree_build(par, prefix_len, mask)
+        sets.append((par, torch.tensor(drafts, **i32), torch.from_numpy(logits).to(dev), mask))
+    tok = torch.zeros((B, T), **i32)
+    acc_idx = torch.zeros((B, 8), **i32)
+    acc_len = torch.zeros(B, **i32)
+    nxt = torch.zeros(B, **i32)
+    new_len = torch.zeros(B, **i32)
+    status = torch.zeros(1, **i32)
+    desc = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0])
+    ws = sv.alloc_attn_workspace(desc, dev)
+    launches_per_step = L + 2
+
+    def attn_layers(i):
+        par, drf, lg, mask = sets[i % N_INPUT_SETS]
+        for l in range(L):
+            sv.specvlm_tree_verify_attn(q[l], k_cache[l], v_cache[l], prefix_len, par, mask, out[l],
+                                        workspace=ws, status=status, desc=desc)
+
+    def tail(i):
+        par, drf, lg, mask = sets[i % N_INPUT_SETS]
+        sv.specvlm_argmax(lg, tok)
+        sv.specvlm_accept_compact(drf, par, tok, k_cache, v_cache, prefix_len, acc_idx, acc_len, nxt, new_len,
+                                  status)
+
+    # The launches of one step are captured once per input set into CUDA graphs (the L
+    # attention launches and the argmax + accept/compact tail separately, so that events
+    # between the two replays time the attention launches); the timed loop replays them.
+    for i in range(N_INPUT_SETS):
+        attn_layers(i)
+        tail(i)
+    torch.cuda.synchronize()
+    graphs = []
+    if not args.no_graph:
+        for i in range(N_INPUT_SETS):
+            ga, gt = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+            with torch.cuda.graph(ga):
+                attn_layers(i)
+            with torch.cuda.graph(gt):
+                tail(i)
+            graphs.append((ga, gt))
+
+    def step(i, ev=None):
+        if ev is not None:
+            ev[0].record()
+        if graphs:
+            graphs[i % N_INPUT_SETS][0].replay()
+        else:
+            attn_layers(i)
+        if ev is not None:
+            ev[1].record()
+        if graphs:
+            graphs[i % N_INPUT_SETS][1].replay()
+        else:
+            tail(i)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    attn_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record()
+    for i in range(args.steps):
+        step(i, attn_events[i])
+    e1.record()
+    sampler.sample()
+    barrier()
+    sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    attn_ms = sum(a.elapsed_time(b) for a, b in attn_events)
+    assert status.item() == 0, f"device status word = {status.item()}"
+
+    # ---- end-to-end: per-step inputs come from pinned host memory, results go back
+    pin = dict(pin_memory=True)
+    h_q = torch.empty((L, B, H, T, D), dtype=torch.bfloat16, **pin).copy_(q)
+    h_tk = torch.empty((L, B, H, T, D), dtype=torch.bfloat16, **pin).normal_()
+    h_tv = torch.empty((L, B, H, T, D), dtype=torch.bfloat16, **pin).normal_()
+    h_sets = [(torch.from_numpy(p).pin_memory(), torch.from_numpy(d).pin_memory(), torch.from_numpy(lg).pin_memory())
+              for p, d, lg in sets_host]
+    h_out = torch.empty((L, B, H, T, D), dtype=torch.bfloat16, **pin)
+    h_res = [torch.empty((B, 8), dtype=torch.int32, **pin)] + [torch.empty(B, dtype=torch.int32, **pin)
+                                                                for _ in range(3)]
+    d_tk, d_tv = torch.empty_like(q), torch.empty_like(q)
+    d_par, d_drf = torch.zeros((B, T), **i32), torch.zeros((B, T), **i32)
+    d_lg = torch.empty((B, T, V), dtype=torch.float32, device=dev)
+    d_mask = torch.zeros((B, T), dtype=torch.int64, device=dev)
+    d_res = [torch.zeros((B, 8), **i32)] + [torch.zeros(B, **i32) for _ in range(3)]
+    same_prefix = bool((P_host == P_host[0]).all())
+    h2d = 3 * h_q.numel() * 2 + 2 * B * T * 4 + B * T * V * 4
+    d2h = h_out.numel() * 2 + sum(t.numel() for t in h_res) * 4
+
+    def e2e_step(i):
+        hp, hd, hl = h_sets[i % N_INPUT_SETS]
+        q.copy_(h_q, non_blocking=True)
+        d_tk.copy_(h_tk, non_blocking=True)
+        d_tv.copy_(h_tv, non_blocking=True)
+        d_par.copy_(hp, non_blocking=True)
+        d_drf.copy_(hd, non_blocking=True)
+        d_lg.copy_(hl, non_blocking=True)
+        # the tree's new K/V rows go to cache slots P_b .. P_b + T - 1 (device-side placement)
+        if same_prefix:
+            p0 = int(P_host[0])
+            k_cache[:, :, :, p0:p0 + T, :].copy_(d_tk)
+            v_cache[:, :, :, p0:p0 + T, :].copy_(d_tv)
+        else:
+            for b in range(B):
+                pb = int(P_host[b])
+                k_cache[:, b, :, pb:pb + T, :].copy_(d_tk[:, b])
+                v_cache[:, b, :, pb:pb + T, :].copy_(d_tv[:, b])
+        sv.specvlm_tree_build(d_par, prefix_len, d_mask)
+        for l in range(L):
+            sv.specvlm_tree_verify_attn(q[l], k_cache[l], v_cache[l], prefix_len, d_par, d_mask, out[l],
+                                        workspace=ws, status=status, desc=desc)
+        sv.specvlm_argmax(d_lg, tok)
+        sv.specvlm_accept_compact(d_drf, d_par, tok, k_cache, v_cache, prefix_len, d_res[0], d_res[1],
+                                  d_res[2], d_res[3], status)
+        h_out.copy_(out, non_blocking=True)
+        for h_t, d_t in zip(h_res, d_res):
+            h_t.copy_(d_t, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 50))
+    for i in range(2):
+        e2e_step(i)
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    f1.record()
+    barrier()
+    e2e_ms = f0.elapsed_time(f1)
+
+    if world > 1:
+        t = torch.tensor([ms_total, attn_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, attn_ms, e2e_ms = (float(x) for x in t.tolist())
+
+    if rank == 0:
+        peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(peaks_path):
+            peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        else:
+            peak, peak_src = 6650.0, "fallback (6.65 TB/s)"
+        kv_bytes_per_launch = float(sum(H * (int(p) + T) * 2 * D * 2 for p in P_host))
+        attn_s_per_launch = attn_ms * 1e-3 / (args.steps * L)
+        achieved = kv_bytes_per_launch / attn_s_per_launch / 1e9
+        traffic = None
+        prof = os.path.join(ROOT, "profiles", "attn_traffic.json")
+        if os.path.exists(prof):
+            try:
+                traffic = json.load(open(prof)).get(cfg.name)
+            except Exception:
+                traffic = None
+        line = {
+            "metric": METRIC, "value": world * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": workload_config(cfg),
+            "attn_us_per_layer": attn_s_per_launch * 1e6, "attn_hbm_gbs": achieved,
+            "attn_frac_of_8tbs_nominal": achieved / 8000.0,
+            "roofline": {"bound": "hbm", "kernel": "tree_verify_attn", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                         "bytes_per_launch": kv_bytes_per_launch},
+            "e2e": {"value": world * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": launches_per_step * args.steps, "launch_mode": "cuda_graph" if graphs else "python",
+            "clocks": sampler.summary(),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            piece, cores = oracle_sample(cfg, 2 if L >= 2 else 1)
+            line["cpu_baseline"] = {
+                "value": 1.0 / piece["est_step_s"], "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": (f"oracle on {2 if L >= 2 else 1} of {L} layers (all sequence-heads) + full argmax/accept + "
+                           f"compaction of those layers, {piece['measured_s']:.1f} s measured; attention and "
+                           f"compaction scaled to {L} layers")}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of CUDA graphs")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = wl.get_config(args.workload)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,204 @@
+/*
+ * specvlm.h -- C ABI of the B200 (sm_100a) tree-verification library.
+ *
+ * The library implements the target model's verification step of EAGLE-2-style
+ * speculative decoding for LLaVA-class VLMs, as the SpecVLM paper uses it:
+ *   - Section 3.1: the target verifies all drafted tokens in one forward pass and
+ *     incorrect tokens are discarded;
+ *   - Section 3.3 (a): the target's latest token is the root of the draft token tree;
+ *   - Section 4.1: the draft is verified with tree attention (top-k 10, 60 tokens);
+ *   - Section 3.2: attention streams the whole (visual-token dominated) KV cache from
+ *     HBM on every step -- the cost this library is built around;
+ *   - abstract / Section 4.1: decoding is lossless with respect to the target.
+ *
+ * Conventions
+ *   - All pointers are DEVICE pointers owned by the caller unless the parameter name
+ *     ends in `_host`. The library allocates no device memory. Scratch memory is a
+ *     caller-provided `workspace` sized by the matching *_workspace_bytes() call and
+ *     zero-filled ONCE (specvlm_workspace_init) before first use; calls leave it ready
+ *     for the next call. Two calls that use the same workspace must not overlap on the
+ *     GPU.
+ *   - Every call only enqueues work on `stream` (a cudaStream_t passed as void*) and
+ *     returns; nothing synchronises.
+ *   - Return value: SPECVLM_OK or a negative SPECVLM_ERR_* detected on the host before
+ *     anything is launched; specvlm_last_error_string() describes the last error of the
+ *     calling thread.
+ *   - Device-side data problems (bad prefix length, malformed tree) never trap: the
+ *     affected sequence is skipped or clamped and SPECVLM_STATUS_* bits are OR-ed into
+ *     the optional `status` word (int32 on the device, may be NULL).
+ *   - Tree layout: T <= 64 nodes, node 0 is the root, parent[0] = -1, parent[i] < i.
+ *     Node t's K/V row lives in cache slot prefix_len[b] + t.
+ *   - Element type of q / k_cache / v_cache / out is bfloat16 (passed as uint16_t bit
+ *     patterns). head_dim D must be 128. Base pointers and all strides must be
+ *     multiples of 8 elements (16 bytes); D is contiguous.
+ */
+#ifndef SPECVLM_H_
+#define SPECVLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPECVLM_VERSION 100
+
+#if defined(__GNUC__)
+#define SPECVLM_API __attribute__((visibility("default")))
+#else
+#define SPECVLM_API
+#endif
+
+#define SPECVLM_OK 0
+#define SPECVLM_ERR_INVALID_ARG (-1)
+#define SPECVLM_ERR_UNSUPPORTED (-2)
+#define SPECVLM_ERR_CUDA (-3)
+#define SPECVLM_ERR_BAD_TREE (-4)
+
+/* bits OR-ed into the device-side status word */
+#define SPECVLM_STATUS_BAD_PREFIX 1  /* prefix_len[b] < 0 or prefix_len[b] + T > S_cap */
+#define SPECVLM_STATUS_BAD_TREE 2    /* parent[0] != -1 or parent[i] outside [0, i)    */
+#define SPECVLM_STATUS_BAD_ACCEPT 4  /* accept_len / accepted_idx out of range         */
+#define SPECVLM_STATUS_TIMEOUT 8     /* a bounded on-chip wait gave up                  */
+
+#define SPECVLM_MAX_TREE 64
+#define SPECVLM_HEAD_DIM 128
+
+/* Shapes and strides (in ELEMENTS) of one layer's attention call. */
+typedef struct specvlm_attn_desc {
+  int32_t B;      /* sequences                                   */
+  int32_t H;      /* heads (multi-head attention: KV heads == H) */
+  int32_t T;      /* tree nodes incl. root, 1..64                */
+  int32_t D;      /* head dim, must be 128                       */
+  int32_t S_cap;  /* cache capacity in token slots per (b, h)    */
+  int32_t num_splits; /* KV splits per (b, h); 0 = library chooses */
+  float softmax_scale; /* 0 = 1/sqrt(D)                          */
+  int32_t reserved;
+  int64_t q_stride_b, q_stride_h, q_stride_t; /* q  [B][H][T][D] by default */
+  int64_t k_stride_b, k_stride_h, k_stride_s; /* K  [B][H][S_cap][D]        */
+  int64_t v_stride_b, v_stride_h, v_stride_s; /* V  [B][H][S_cap][D]        */
+  int64_t o_stride_b, o_stride_h, o_stride_t; /* out [B][H][T][D]           */
+} specvlm_attn_desc;
+
+/* Shapes and strides (in ELEMENTS) of the multi-layer KV cache for compaction. */
+typedef struct specvlm_kv_desc {
+  int32_t L, B, H, S_cap, D; /* D must be 128 */
+  int32_t reserved;
+  int64_t stride_l, stride_b, stride_h, stride_s; /* same for K and V */
+} specvlm_kv_desc;
+
+SPECVLM_API int specvlm_version(void);
+SPECVLM_API const char* specvlm_last_error_string(void);
+
+/* Bytes of scratch specvlm_tree_verify_attn needs for this descriptor (split-KV partial
+ * results and arrival counters). Host call. */
+SPECVLM_API int specvlm_attn_workspace_bytes(const specvlm_attn_desc* desc_host, size_t* bytes_host);
+
+/* Zero-fill a workspace (once, after allocating it). */
+SPECVLM_API int specvlm_workspace_init(void* workspace, size_t bytes, void* stream);
+
+/*
+ * Tree metadata (tree attention, Section 4.1; root, Section 3.3 (a)).
+ *   tree_parent   int32 [B][T]
+ *   prefix_len    int32 [B]
+ *   mask_bits     uint64 [B][T] out: bit t of mask_bits[b][i] set iff t is i or an
+ *                 ancestor of i
+ *   depth         int32 [B][T] out (may be NULL): edges from the root
+ *   pos           int32 [B][T] out (may be NULL): prefix_len[b] + depth (position id)
+ * A malformed tree sets SPECVLM_STATUS_BAD_TREE and yields self-only masks.
+ */
+SPECVLM_API int specvlm_tree_build(const int32_t* tree_parent, const int32_t* prefix_len, int B, int T,
+                       uint64_t* mask_bits, int32_t* depth, int32_t* pos, int32_t* status,
+                       void* stream);
+
+/* Host-side validation of one tree (host pointers): parent[0] = -1, parent[i] in [0, i),
+ * T in 1..64, and (if draft_tokens_host != NULL) siblings carry distinct tokens.
+ * Returns SPECVLM_OK or SPECVLM_ERR_BAD_TREE. */
+SPECVLM_API int specvlm_tree_validate_host(const int32_t* tree_parent_host, const int32_t* draft_tokens_host,
+                               int T);
+
+/*
+ * Tree-verification attention for ONE layer (Sections 3.1, 3.2, 4.1).
+ * For each sequence b, head h and tree node i < T:
+ *     out[b][h][i][:] = softmax_j( q[b][h][i] . K[b][h][j] * scale ) V[b][h][j][:]
+ * over keys j < prefix_len[b] (all visible) and j = prefix_len[b] + t, t < T, visible
+ * iff bit t of tree_mask_bits[b][i] is set. Slots >= prefix_len[b] + T are never read
+ * into the result (they may hold any bit pattern). A node with no visible key gets zeros.
+ *   q, out            bf16, strides from desc
+ *   k_cache, v_cache  bf16, this layer's cache, strides from desc; read-only here
+ *   prefix_len        int32 [B]
+ *   tree_parent       int32 [B][T]; used only when tree_mask_bits == NULL (the mask is
+ *                     then derived from it); may be NULL otherwise
+ *   tree_mask_bits    uint64 [B][T] or NULL
+ *   workspace         from specvlm_attn_workspace_bytes, zero-initialised once
+ * bf16 inputs, fp32 accumulation, bf16 output.
+ */
+SPECVLM_API int specvlm_tree_verify_attn(const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache,
+                             const int32_t* prefix_len, const int32_t* tree_parent,
+                             const uint64_t* tree_mask_bits, uint16_t* out,
+                             const specvlm_attn_desc* desc_host, void* workspace,
+                             int32_t* status, void* stream);
+
+/*
+ * Greedy target token per tree node (temperature 0; "negligible" sampling cost of
+ * Eq. 1): argmax_tokens[b][i] = argmax_v target_logits[b][i][v]; ties -> lowest v;
+ * -0 == +0; inputs must be NaN-free.
+ *   target_logits  fp32, row r = b*T + i starts at target_logits + r * row_stride
+ *                  (row_stride in elements, multiple of 4, >= V)
+ *   argmax_tokens  int32 [B][T] out
+ */
+SPECVLM_API int specvlm_argmax(const float* target_logits, int B, int T, int V, int64_t row_stride,
+                   int32_t* argmax_tokens, void* stream);
+
+/*
+ * Lossless temperature-0 acceptance (Section 3.1: incorrect tokens are discarded;
+ * abstract: lossless). Node i > 0 is kept iff draft_tokens[i] equals the target's greedy
+ * token at parent[i] and its parent is kept; the root is always kept. The result is the
+ * deepest kept node (lowest index among equals) and its root path.
+ *   draft_tokens   int32 [B][T]   (entry 0 = root token, unused by the rule)
+ *   tree_parent    int32 [B][T]
+ *   target_logits  fp32 [B][T][V] contiguous rows (row stride V), or NULL
+ *   argmax_tokens  int32 [B][T]: input when target_logits == NULL; otherwise written
+ *                  by an argmax pass first (must be non-NULL in both cases)
+ *   accepted_idx   int32 [B][acc_stride] out: node indices of the kept path, entry 0 = 0;
+ *                  unused entries = -1; acc_stride >= 1; only the first acc_stride path
+ *                  entries are written
+ *   accept_len     int32 [B] out: kept DRAFTED tokens (root and bonus token not counted)
+ *   next_token     int32 [B] out: the target's greedy token at the last kept node
+ */
+SPECVLM_API int specvlm_accept(const int32_t* draft_tokens, const int32_t* tree_parent,
+                   const float* target_logits, int32_t* argmax_tokens, int B, int T, int V,
+                   int32_t* accepted_idx, int acc_stride, int32_t* accept_len,
+                   int32_t* next_token, int32_t* status, void* stream);
+
+/*
+ * KV compaction after acceptance (the KV cache is the resource the paper's cost model
+ * is about, Sections 1 and 3.2). For every layer, for K and V, for every (b, h) and
+ * j = 1..accept_len[b]: the 256-byte row in slot prefix_len[b] + accepted_idx[b][j] moves
+ * to slot prefix_len[b] + j, in place; all sources of one (layer, b, h) are read before
+ * any destination is written. Every other byte of the caches is left untouched.
+ * new_prefix_len[b] = prefix_len[b] + 1 + accept_len[b]; it must NOT alias prefix_len.
+ */
+SPECVLM_API int specvlm_kv_compact(uint16_t* k_cache, uint16_t* v_cache, const specvlm_kv_desc* desc_host,
+                       const int32_t* prefix_len, const int32_t* accepted_idx, int acc_stride,
+                       const int32_t* accept_len, int32_t* new_prefix_len, int32_t* status,
+                       void* stream);
+
+/*
+ * Fused path walk + KV gather: specvlm_accept (from argmax_tokens) and specvlm_kv_compact
+ * in ONE kernel launch. Every thread block redoes the <= 64-node walk, then moves its share
+ * of rows; block 0 also writes accepted_idx / accept_len / next_token / new_prefix_len.
+ * Arguments as in the two calls above (argmax_tokens is an input here).
+ */
+SPECVLM_API int specvlm_accept_compact(const int32_t* draft_tokens, const int32_t* tree_parent,
+                           const int32_t* argmax_tokens, int T, uint16_t* k_cache,
+                           uint16_t* v_cache, const specvlm_kv_desc* desc_host,
+                           const int32_t* prefix_len, int32_t* accepted_idx, int acc_stride,
+                           int32_t* accept_len, int32_t* next_token, int32_t* new_prefix_len,
+                           int32_t* status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECVLM_H_ */
