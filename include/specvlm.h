@@ -141,6 +141,33 @@ SPECVLM_API int specvlm_tree_verify_attn(const uint16_t* q, const uint16_t* k_ca
                              int32_t* status, void* stream);
 
 /*
+ * Same computation and arguments as specvlm_tree_verify_attn, minus the workspace: the
+ * split-KV scratch is a fixed array inside the library (about 16.3 MiB of device memory per
+ * GPU, held from the moment the library is loaded on that GPU until the process exits).
+ * The paper has no counterpart for this call; it exists for callers that cannot allocate
+ * device memory when they need attention: engines whose memory pool already owns all of
+ * HBM, decode loops that must avoid the device-wide stall of an allocation, plug-ins that
+ * receive raw pointers and no allocator. The call itself allocates nothing and frees
+ * nothing.
+ *   - Limits: B*H <= 1024 and B*H*splits <= 512, where splits is desc.num_splits or, if
+ *     that is 0, the library's choice for the shape. Beyond them the call returns
+ *     SPECVLM_ERR_UNSUPPORTED with a message that states the numbers; set desc.num_splits
+ *     lower or use the workspace variant.
+ *   - The first call on each device looks up the array's device address and raises the
+ *     kernel's shared-memory limit; make that first call outside any stream capture, with
+ *     the device current.
+ *   - All calls on one GPU share the one array. It keeps the previous call's contents; the
+ *     call clears the part that must start at zero on `stream` before the kernel runs. Two
+ *     calls that overlap on the GPU (different streams, no ordering) race on the array and
+ *     give wrong results: order them.
+ */
+SPECVLM_API int specvlm_tree_verify_attn_static(const uint16_t* q, const uint16_t* k_cache,
+                                    const uint16_t* v_cache, const int32_t* prefix_len,
+                                    const int32_t* tree_parent, const uint64_t* tree_mask_bits,
+                                    uint16_t* out, const specvlm_attn_desc* desc_host,
+                                    int32_t* status, void* stream);
+
+/*
  * Greedy target token per tree node (temperature 0; "negligible" sampling cost of
  * Eq. 1): argmax_tokens[b][i] = argmax_v target_logits[b][i][v]; ties -> lowest v;
  * -0 == +0; inputs must be NaN-free.

@@ -28,6 +28,7 @@ EXPORTS = (
     "specvlm_tree_build",
     "specvlm_tree_validate_host",
     "specvlm_tree_verify_attn",
+    "specvlm_tree_verify_attn_static",
     "specvlm_argmax",
     "specvlm_accept",
     "specvlm_kv_compact",
@@ -89,6 +90,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.specvlm_tree_validate_host.argtypes = [vp, vp, i32]
     lib.specvlm_tree_verify_attn.restype = i32
     lib.specvlm_tree_verify_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(AttnDesc), vp, vp, vp]
+    lib.specvlm_tree_verify_attn_static.restype = i32
+    lib.specvlm_tree_verify_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(AttnDesc), vp, vp]
     lib.specvlm_argmax.restype = i32
     lib.specvlm_argmax.argtypes = [vp, i32, i32, i32, i64, vp, vp]
     lib.specvlm_accept.restype = i32
@@ -212,6 +215,28 @@ def specvlm_tree_verify_attn(q: torch.Tensor, k_cache: torch.Tensor, v_cache: to
     _check(load_library().specvlm_tree_verify_attn(
         _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(prefix_len), _ptr(tree_parent), _ptr(tree_mask_bits),
         _ptr(out), ctypes.byref(desc), _ptr(workspace), _ptr(status), _stream()))
+
+
+def specvlm_tree_verify_attn_static(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                                    prefix_len: torch.Tensor, tree_parent: Optional[torch.Tensor],
+                                    tree_mask_bits: Optional[torch.Tensor], out: torch.Tensor,
+                                    status: Optional[torch.Tensor] = None, num_splits: int = 0,
+                                    softmax_scale: float = 0.0, desc: Optional[AttnDesc] = None) -> None:
+    """Attention for callers that have no device memory to spare for a workspace (a memory pool
+    that already owns the GPU, a decode loop that must not stall on an allocation): the split-KV
+    scratch is a fixed array inside the library. Same results as specvlm_tree_verify_attn. Shapes
+    beyond the built-in limits (B*H <= 1024, B*H*splits <= 512) raise SpecvlmError. Calls share
+    the array, so calls that overlap on the GPU must be ordered by the caller."""
+    if desc is None:
+        desc = make_attn_desc(q, k_cache, v_cache, out, num_splits, softmax_scale)
+    _need(prefix_len, torch.int32, "prefix_len")
+    if tree_mask_bits is not None:
+        _need(tree_mask_bits, _MASK_DTYPES, "tree_mask_bits")
+    if tree_parent is not None:
+        _need(tree_parent, torch.int32, "tree_parent")
+    _check(load_library().specvlm_tree_verify_attn_static(
+        _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(prefix_len), _ptr(tree_parent), _ptr(tree_mask_bits),
+        _ptr(out), ctypes.byref(desc), _ptr(status), _stream()))
 
 
 def specvlm_argmax(target_logits: torch.Tensor, argmax_tokens: torch.Tensor) -> None:

@@ -14,6 +14,8 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
+#include <mutex>
+
 namespace specvlm {
 
 constexpr int kD = SPECVLM_HEAD_DIM;  // 128
@@ -451,4 +453,100 @@ extern "C" int specvlm_tree_verify_attn(const uint16_t* q, const uint16_t* k_cac
   dim3 grid(splits, desc->H, desc->B);
   tree_attn_mma_kernel<<<grid, kThreads, kSmemBytes, static_cast<cudaStream_t>(stream)>>>(p);
   return check_cuda(cudaGetLastError(), "tree_verify_attn launch");
+}
+
+// ---------------------------------------------------------------------------------------------
+// Variant of the split-KV attention call that needs no scratch memory from the caller.
+//
+// Who it is for: callers that cannot obtain device memory at the point of the call. Typical
+// cases are a serving engine that handed the whole of HBM to its KV-cache block pool at
+// start-up (a later cudaMalloc fails or forces the pool to shrink), a decode loop that must not
+// take the device-wide synchronisation an allocation implies, and plug-in code that is given
+// raw input/output pointers but no allocator. For them the split-KV partials and arrival
+// counters live in the fixed device array below, which every GPU that loads this library keeps
+// until the process exits.
+namespace specvlm {
+
+constexpr int kStaticMaxBH = 1024;     // sequences x heads
+constexpr int kStaticMaxUnits = 512;   // sequences x heads x splits
+constexpr size_t kStaticCounterBytes = kStaticMaxBH * sizeof(int32_t);
+constexpr size_t kStaticMlBytes = static_cast<size_t>(kStaticMaxUnits) * kRows * 2 * sizeof(float);
+constexpr size_t kStaticOBytes = static_cast<size_t>(kStaticMaxUnits) * kRows * kD * sizeof(float);
+constexpr size_t kStaticBytes = kStaticCounterBytes + kStaticMlBytes + kStaticOBytes;  // ~16.3 MiB
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address; the
+// address a kernel may use comes from cudaGetSymbolAddress, asked once per device with that
+// device current.
+static int static_scratch_address(unsigned char** out) {
+  static unsigned char* addr[64] = {};
+  static std::mutex mu;
+  int dev = 0;
+  int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
+  if (rc != SPECVLM_OK) return rc;
+  if (dev < 0 || dev >= 64) return fail(SPECVLM_ERR_UNSUPPORTED, "static scratch: device index out of range");
+  std::lock_guard<std::mutex> lock(mu);
+  if (addr[dev] == nullptr) {
+    void* p = nullptr;
+    rc = check_cuda(cudaGetSymbolAddress(&p, g_static_scratch), "cudaGetSymbolAddress(static scratch)");
+    if (rc != SPECVLM_OK) return rc;
+    if (p == nullptr) return fail(SPECVLM_ERR_CUDA, "static scratch: null symbol address");
+    rc = check_cuda(cudaFuncSetAttribute(tree_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kSmemBytes),
+                    "attn smem attribute");
+    if (rc != SPECVLM_OK) return rc;
+    addr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = addr[dev];
+  return SPECVLM_OK;
+}
+
+}  // namespace specvlm
+
+extern "C" int specvlm_tree_verify_attn_static(const uint16_t* q, const uint16_t* k_cache,
+                                               const uint16_t* v_cache, const int32_t* prefix_len,
+                                               const int32_t* tree_parent, const uint64_t* tree_mask_bits,
+                                               uint16_t* out, const specvlm_attn_desc* desc, int32_t* status,
+                                               void* stream) {
+  int rc = check_attn_desc(desc);
+  if (rc != SPECVLM_OK) return rc;
+  if (desc->B == 0) return SPECVLM_OK;
+  SPECVLM_REQUIRE(q && k_cache && v_cache && prefix_len && out, "tree_verify_attn_static: null pointer");
+  SPECVLM_REQUIRE(tree_mask_bits != nullptr || tree_parent != nullptr,
+                  "tree_verify_attn_static: need tree_mask_bits or tree_parent");
+  SPECVLM_REQUIRE(aligned16(q) && aligned16(k_cache) && aligned16(v_cache) && aligned16(out),
+                  "tree_verify_attn_static: q/k/v/out must be 16-byte aligned");
+  const int splits = resolve_num_splits(*desc);
+  const int64_t bh = static_cast<int64_t>(desc->B) * desc->H;
+  if (bh > kStaticMaxBH || bh * splits > kStaticMaxUnits)
+    return fail(SPECVLM_ERR_UNSUPPORTED,
+                "tree_verify_attn_static: B*H = " + std::to_string(bh) + " with " + std::to_string(splits) +
+                    " KV splits exceeds the built-in scratch (limits: B*H <= " + std::to_string(kStaticMaxBH) +
+                    ", B*H*splits <= " + std::to_string(kStaticMaxUnits) +
+                    "); lower desc.num_splits or use specvlm_tree_verify_attn with a workspace");
+  unsigned char* scratch = nullptr;
+  rc = static_scratch_address(&scratch);
+  if (rc != SPECVLM_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The array keeps whatever the previous call left; the arrival counters must start at zero.
+  rc = check_cuda(cudaMemsetAsync(scratch, 0, kStaticCounterBytes, s), "static scratch counter clear");
+  if (rc != SPECVLM_OK) return rc;
+
+  AttnParams p;
+  p.q = q; p.k = k_cache; p.v = v_cache; p.out = out;
+  p.prefix_len = prefix_len; p.parent = tree_parent; p.mask = tree_mask_bits; p.status = status;
+  p.counters = reinterpret_cast<int32_t*>(scratch);
+  p.part_ml = reinterpret_cast<float*>(scratch + kStaticCounterBytes);
+  p.part_o = reinterpret_cast<float*>(scratch + kStaticCounterBytes + kStaticMlBytes);
+  p.B = desc->B; p.H = desc->H; p.T = desc->T; p.S_cap = desc->S_cap; p.splits = splits;
+  const float scale = desc->softmax_scale > 0.f ? desc->softmax_scale : 1.0f / sqrtf(static_cast<float>(kD));
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.q_sb = desc->q_stride_b; p.q_sh = desc->q_stride_h; p.q_st = desc->q_stride_t;
+  p.k_sb = desc->k_stride_b; p.k_sh = desc->k_stride_h; p.k_ss = desc->k_stride_s;
+  p.v_sb = desc->v_stride_b; p.v_sh = desc->v_stride_h; p.v_ss = desc->v_stride_s;
+  p.o_sb = desc->o_stride_b; p.o_sh = desc->o_stride_h; p.o_st = desc->o_stride_t;
+  dim3 grid(splits, desc->H, desc->B);
+  tree_attn_mma_kernel<<<grid, kThreads, kSmemBytes, s>>>(p);
+  return check_cuda(cudaGetLastError(), "tree_verify_attn_static launch");
 }
