@@ -11,6 +11,7 @@
 // that arrives last (atomic counter, no waiting) combines them and writes bf16.
 #include "common.cuh"
 
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -95,8 +96,11 @@ __device__ __forceinline__ void load_tile(uint32_t sk, uint32_t sv, const uint16
   }
 }
 
-__global__ void __launch_bounds__(kThreads)
-tree_attn_mma_kernel(const AttnParams p) {
+// kClusterCombine = false: splits meet through the global workspace (any split count).
+// kClusterCombine = true : the splits of one (sequence, head) form a thread-block cluster
+// (cluster size == split count <= 8) and meet through distributed shared memory.
+template <bool kClusterCombine>
+__device__ __forceinline__ void tree_attn_body(const AttnParams& p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t sq = smem_u32(smem);
   const uint32_t stage0 = sq + kRows * kD * 2;
@@ -300,6 +304,62 @@ tree_attn_mma_kernel(const AttnParams p) {
     return;
   }
 
+  if constexpr (kClusterCombine) {
+    // ---- partial into this CTA's own shared memory (the K/V stages are free now)
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    __syncthreads();  // every warp is done reading the stages
+    float* so = reinterpret_cast<float*>(smem + kRows * kD * 2);  // [64][128] fp32
+    float* sml = so + kRows * kD;                                 // [64][2]
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      *reinterpret_cast<float2*>(so + row0 * kD + i * 8 + t4 * 2) = make_float2(o[i][0], o[i][1]);
+      *reinterpret_cast<float2*>(so + row1 * kD + i * 8 + t4 * 2) = make_float2(o[i][2], o[i][3]);
+    }
+    if (t4 == 0) {
+      *reinterpret_cast<float2*>(sml + row0 * 2) = make_float2(m0, l0);
+      *reinterpret_cast<float2*>(sml + row1 * 2) = make_float2(m1, l1);
+    }
+    cluster.sync();  // all partials of this (sequence, head) are visible cluster-wide
+    // Rows are dealt round-robin to the cluster's CTAs, then to the CTA's warps; a lane owns
+    // four output columns and reads them from every CTA's shared memory.
+    uint16_t* obase = p.out + b * p.o_sb + h * p.o_sh;
+    const int nsplit = p.splits;  // == cluster size
+    int nth = 0;
+    for (int row = split; row < T; row += nsplit, ++nth) {
+      if ((nth & 3) != warp) continue;
+      float2 ml = make_float2(-INFINITY, 0.f);
+      if (lane < nsplit) ml = *reinterpret_cast<const float2*>(cluster.map_shared_rank(sml, lane) + row * 2);
+      float mstar = ml.x;
+#pragma unroll
+      for (int off = 4; off > 0; off >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, off));
+      const float w = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mstar);
+      float lsum = w * ml.y;
+#pragma unroll
+      for (int off = 4; off > 0; off >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, off);
+      lsum = __shfl_sync(0xffffffffu, lsum, 0);
+      float4 x[8];
+#pragma unroll
+      for (int s = 0; s < 8; ++s)
+        if (s < nsplit) x[s] = *(reinterpret_cast<const float4*>(cluster.map_shared_rank(so, s) + row * kD) + lane);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        const float ws = __shfl_sync(0xffffffffu, w, s);
+        if (s < nsplit && ws > 0.f) {
+          acc.x += ws * x[s].x; acc.y += ws * x[s].y; acc.z += ws * x[s].z; acc.w += ws * x[s].w;
+        }
+      }
+      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+      uint2 packed;
+      packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+      packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+      *reinterpret_cast<uint2*>(obase + row * p.o_st + lane * 4) = packed;
+    }
+    cluster.sync();  // nobody leaves while its shared memory may still be read
+    return;
+  }
+
   // ---- write this split's partial (unnormalised O, running max, running sum)
   {
     float* po = p.part_o + (static_cast<int64_t>(bh) * p.splits + split) * kRows * kD;
@@ -358,19 +418,34 @@ tree_attn_mma_kernel(const AttnParams p) {
   }
 }
 
+__global__ void __launch_bounds__(kThreads) tree_attn_mma_kernel(const AttnParams p) {
+  tree_attn_body<false>(p);
+}
+
+__global__ void __launch_bounds__(kThreads) tree_attn_mma_cluster_kernel(const AttnParams p) {
+  tree_attn_body<true>(p);
+}
+
+constexpr int kMaxClusterSplits = 8;  // portable cluster size limit
+
 int resolve_num_splits(const specvlm_attn_desc& d) {
   const int max_tiles = (d.S_cap + kTileN - 1) / kTileN;
   int splits = d.num_splits;
   if (splits <= 0) {
+    // about two CTAs per SM; up to twice the cluster limit is folded onto the cluster path
     const int64_t bh = static_cast<int64_t>(d.B) * d.H;
     const int64_t target = 2 * static_cast<int64_t>(sm_count());
     splits = static_cast<int>((target + bh - 1) / (bh > 0 ? bh : 1));
+    if (splits > kMaxClusterSplits && splits <= 2 * kMaxClusterSplits) splits = kMaxClusterSplits;
   }
   if (splits > max_tiles) splits = max_tiles;
   if (splits > 64) splits = 64;
   if (splits < 1) splits = 1;
   return splits;
 }
+
+// Split counts up to the portable cluster size combine on chip and need no workspace.
+static bool uses_cluster(int splits) { return splits >= 2 && splits <= kMaxClusterSplits; }
 
 static int check_attn_desc(const specvlm_attn_desc* d) {
   SPECVLM_REQUIRE(d != nullptr, "attn desc is null");
@@ -403,7 +478,10 @@ extern "C" int specvlm_attn_workspace_bytes(const specvlm_attn_desc* desc, size_
   SPECVLM_REQUIRE(bytes != nullptr, "attn_workspace_bytes: null result pointer");
   const size_t splits = resolve_num_splits(*desc);
   const size_t bh = static_cast<size_t>(desc->B) * desc->H;
-  *bytes = counters_bytes(*desc) + bh * splits * kRows * 2 * sizeof(float) + bh * splits * kRows * kD * sizeof(float);
+  if (splits == 1 || uses_cluster(static_cast<int>(splits)))
+    *bytes = 0;
+  else
+    *bytes = counters_bytes(*desc) + bh * splits * kRows * 2 * sizeof(float) + bh * splits * kRows * kD * sizeof(float);
   return SPECVLM_OK;
 }
 
@@ -421,8 +499,9 @@ extern "C" int specvlm_tree_verify_attn(const uint16_t* q, const uint16_t* k_cac
   SPECVLM_REQUIRE(aligned16(q) && aligned16(k_cache) && aligned16(v_cache) && aligned16(out),
                   "tree_verify_attn: q/k/v/out must be 16-byte aligned");
   const int splits = resolve_num_splits(*desc);
-  SPECVLM_REQUIRE(splits == 1 || (workspace != nullptr && aligned16(workspace)),
-                  "tree_verify_attn: workspace required (16-byte aligned) when KV is split");
+  const bool cluster = uses_cluster(splits);
+  SPECVLM_REQUIRE(splits == 1 || cluster || (workspace != nullptr && aligned16(workspace)),
+                  "tree_verify_attn: workspace required (16-byte aligned) when KV is split more than 8 ways");
 
   AttnParams p;
   p.q = q; p.k = k_cache; p.v = v_cache; p.out = out;
@@ -448,9 +527,28 @@ extern "C" int specvlm_tree_verify_attn(const uint16_t* q, const uint16_t* k_cac
     rc = check_cuda(cudaFuncSetAttribute(tree_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes),
                     "attn smem attribute");
     if (rc != SPECVLM_OK) return rc;
+    rc = check_cuda(cudaFuncSetAttribute(tree_attn_mma_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kSmemBytes),
+                    "attn smem attribute (cluster)");
+    if (rc != SPECVLM_OK) return rc;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   dim3 grid(splits, desc->H, desc->B);
+  if (cluster) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = splits;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return check_cuda(cudaLaunchKernelEx(&cfg, tree_attn_mma_cluster_kernel, p), "tree_verify_attn cluster launch");
+  }
   tree_attn_mma_kernel<<<grid, kThreads, kSmemBytes, static_cast<cudaStream_t>(stream)>>>(p);
   return check_cuda(cudaGetLastError(), "tree_verify_attn launch");
 }

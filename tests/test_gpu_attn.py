@@ -265,14 +265,14 @@ def test_output_rows_beyond_tree_and_neighbours_untouched():
 
 
 def test_invalid_arguments_are_rejected_on_the_host():
-    q, k, v, pl, parents, masks = make_case(19, B=1, H=2, T=26, prefixes=[64])
+    q, k, v, pl, parents, masks = make_case(19, B=1, H=2, T=26, prefixes=[1000])
     qt, kt, vt = bits_to_torch(q), bits_to_torch(k), bits_to_torch(v)
     out = torch.empty_like(qt)
     plt = torch.tensor(pl, dtype=torch.int32, device="cuda")
     with pytest.raises(sv.SpecvlmError):       # neither mask nor parent
         sv.specvlm_tree_verify_attn(qt, kt, vt, plt, None, None, out, num_splits=1)
-    with pytest.raises(sv.SpecvlmError):       # split without a workspace
-        sv.specvlm_tree_verify_attn(qt, kt, vt, plt, None, mask_to_torch(masks), out, num_splits=2)
+    with pytest.raises(sv.SpecvlmError):       # more than 8 splits without a workspace
+        sv.specvlm_tree_verify_attn(qt, kt, vt, plt, None, mask_to_torch(masks), out, num_splits=12)
     with pytest.raises(sv.SpecvlmError):       # misaligned q (offset by one element)
         flat = torch.empty(qt.numel() + 8, dtype=torch.bfloat16, device="cuda")
         q_bad = flat[1:1 + qt.numel()].view_as(qt)

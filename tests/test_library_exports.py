@@ -53,9 +53,12 @@ def test_host_side_argument_errors_need_no_gpu():
     d.k_stride_h = 12                                          # not a multiple of 8
     assert lib.specvlm_attn_workspace_bytes(ctypes.byref(d), ctypes.byref(n)) == -1
     d.k_stride_h = 1024 * 128
-    d.num_splits = 4
+    d.num_splits = 4                                           # <= 8 splits combine on chip
     assert lib.specvlm_attn_workspace_bytes(ctypes.byref(d), ctypes.byref(n)) == 0
-    assert n.value == 256 + 32 * 4 * 64 * 2 * 4 + 32 * 4 * 64 * 128 * 4
+    assert n.value == 0
+    d.num_splits = 12
+    assert lib.specvlm_attn_workspace_bytes(ctypes.byref(d), ctypes.byref(n)) == 0
+    assert n.value == 256 + 32 * 12 * 64 * 2 * 4 + 32 * 12 * 64 * 128 * 4
     # null pointers are rejected before any launch
     assert lib.specvlm_argmax(None, 1, 60, 32000, 32000, None, None) == -1
     assert lib.specvlm_tree_build(None, None, 1, 60, None, None, None, None, None) == -1
