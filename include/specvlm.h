@@ -62,6 +62,9 @@ extern "C" {
 #define SPECVLM_STATUS_BAD_ACCEPT 4  /* accept_len / accepted_idx out of range         */
 #define SPECVLM_STATUS_TIMEOUT 8     /* a bounded on-chip wait gave up                  */
 
+/* specvlm_attn_desc.flags: run the older mma.sync kernels instead of the tcgen05 kernel */
+#define SPECVLM_ATTN_FLAG_LEGACY_MMA 1
+
 #define SPECVLM_MAX_TREE 64
 #define SPECVLM_HEAD_DIM 128
 
@@ -74,7 +77,7 @@ typedef struct specvlm_attn_desc {
   int32_t S_cap;  /* cache capacity in token slots per (b, h)    */
   int32_t num_splits; /* KV splits per (b, h); 0 = library chooses */
   float softmax_scale; /* 0 = 1/sqrt(D)                          */
-  int32_t reserved;
+  int32_t flags;  /* SPECVLM_ATTN_FLAG_* bits, normally 0        */
   int64_t q_stride_b, q_stride_h, q_stride_t; /* q  [B][H][T][D] by default */
   int64_t k_stride_b, k_stride_h, k_stride_s; /* K  [B][H][S_cap][D]        */
   int64_t v_stride_b, v_stride_h, v_stride_s; /* V  [B][H][S_cap][D]        */

@@ -44,7 +44,7 @@ class AttnDesc(ctypes.Structure):
     _fields_ = [
         ("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("D", ctypes.c_int32),
         ("S_cap", ctypes.c_int32), ("num_splits", ctypes.c_int32),
-        ("softmax_scale", ctypes.c_float), ("reserved", ctypes.c_int32),
+        ("softmax_scale", ctypes.c_float), ("flags", ctypes.c_int32),
         ("q_stride_b", ctypes.c_int64), ("q_stride_h", ctypes.c_int64), ("q_stride_t", ctypes.c_int64),
         ("k_stride_b", ctypes.c_int64), ("k_stride_h", ctypes.c_int64), ("k_stride_s", ctypes.c_int64),
         ("v_stride_b", ctypes.c_int64), ("v_stride_h", ctypes.c_int64), ("v_stride_s", ctypes.c_int64),
@@ -135,8 +135,11 @@ def specvlm_version() -> int:
     return load_library().specvlm_version()
 
 
+ATTN_FLAG_LEGACY_MMA = 1
+
+
 def make_attn_desc(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,
-                   num_splits: int = 0, softmax_scale: float = 0.0) -> AttnDesc:
+                   num_splits: int = 0, softmax_scale: float = 0.0, flags: int = 0) -> AttnDesc:
     """q/out: [B][H][T][D] views, k/v: [B][H][S_cap][D] views (any strides, D contiguous)."""
     B, H, T, D = q.shape
     for name, t in (("q", q), ("k_cache", k_cache), ("v_cache", v_cache), ("out", out)):
@@ -149,7 +152,7 @@ def make_attn_desc(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor
         raise SpecvlmError("out must have q's shape")
     d = AttnDesc()
     d.B, d.H, d.T, d.D, d.S_cap = B, H, T, D, k_cache.shape[2]
-    d.num_splits, d.softmax_scale = num_splits, softmax_scale
+    d.num_splits, d.softmax_scale, d.flags = num_splits, softmax_scale, flags
     d.q_stride_b, d.q_stride_h, d.q_stride_t = q.stride(0), q.stride(1), q.stride(2)
     d.k_stride_b, d.k_stride_h, d.k_stride_s = k_cache.stride(0), k_cache.stride(1), k_cache.stride(2)
     d.v_stride_b, d.v_stride_h, d.v_stride_s = v_cache.stride(0), v_cache.stride(1), v_cache.stride(2)

@@ -10,6 +10,7 @@
 // Splits of one (sequence, head) meet through fp32 partials in the workspace; the split
 // that arrives last (atomic counter, no waiting) combines them and writes bf16.
 #include "common.cuh"
+#include "attn_params.cuh"
 
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
@@ -26,23 +27,6 @@ constexpr int kThreads = 128;         // 4 warps x 16 query rows
 constexpr int kStages = 3;
 constexpr int kTileBytes = kTileN * kD * 2;  // 16 KB
 constexpr int kSmemBytes = kRows * kD * 2 + kStages * 2 * kTileBytes;  // 16 KB + 96 KB
-
-struct AttnParams {
-  const uint16_t* q;
-  const uint16_t* k;
-  const uint16_t* v;
-  uint16_t* out;
-  const int32_t* prefix_len;
-  const int32_t* parent;
-  const uint64_t* mask;
-  int32_t* status;
-  int32_t* counters;  // [B*H]
-  float* part_ml;     // [B*H][splits][64][2]
-  float* part_o;      // [B*H][splits][64][128]
-  int B, H, T, S_cap, splits;
-  float scale_log2;
-  int64_t q_sb, q_sh, q_st, k_sb, k_sh, k_ss, v_sb, v_sh, v_ss, o_sb, o_sh, o_st;
-};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -428,16 +412,29 @@ __global__ void __launch_bounds__(kThreads) tree_attn_mma_cluster_kernel(const A
 
 constexpr int kMaxClusterSplits = 8;  // portable cluster size limit
 
+// The tcgen05 path (attn_tc.cu) takes calls with up to 8 splits unless the descriptor asks for
+// the legacy kernels; everything else runs on the mma.sync kernels in this file.
+static bool wants_legacy(const specvlm_attn_desc& d) { return (d.flags & SPECVLM_ATTN_FLAG_LEGACY_MMA) != 0; }
+
 int resolve_num_splits(const specvlm_attn_desc& d) {
-  const int max_tiles = (d.S_cap + kTileN - 1) / kTileN;
+  const bool legacy = wants_legacy(d);
   int splits = d.num_splits;
+  const int64_t bh = static_cast<int64_t>(d.B) * d.H > 0 ? static_cast<int64_t>(d.B) * d.H : 1;
   if (splits <= 0) {
-    // about two CTAs per SM; up to twice the cluster limit is folded onto the cluster path
-    const int64_t bh = static_cast<int64_t>(d.B) * d.H;
-    const int64_t target = 2 * static_cast<int64_t>(sm_count());
-    splits = static_cast<int>((target + bh - 1) / (bh > 0 ? bh : 1));
-    if (splits > kMaxClusterSplits && splits <= 2 * kMaxClusterSplits) splits = kMaxClusterSplits;
+    if (legacy) {
+      // about two CTAs per SM; up to twice the cluster limit is folded onto the cluster path
+      const int64_t target = 2 * static_cast<int64_t>(sm_count());
+      splits = static_cast<int>((target + bh - 1) / bh);
+      if (splits > kMaxClusterSplits && splits <= 2 * kMaxClusterSplits) splits = kMaxClusterSplits;
+    } else {
+      // one CTA per SM, the splits of a (sequence, head) in one cluster
+      splits = static_cast<int>(sm_count() / bh);
+      if (splits > kMaxClusterSplits) splits = kMaxClusterSplits;
+    }
   }
+  const bool tc_path = !legacy && splits <= kMaxClusterSplits;
+  const int tile = tc_path ? 128 : kTileN;
+  const int max_tiles = (d.S_cap + tile - 1) / tile;
   if (splits > max_tiles) splits = max_tiles;
   if (splits > 64) splits = 64;
   if (splits < 1) splits = 1;
@@ -533,6 +530,9 @@ extern "C" int specvlm_tree_verify_attn(const uint16_t* q, const uint16_t* k_cac
     if (rc != SPECVLM_OK) return rc;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
+  if (!wants_legacy(*desc) && splits <= kMaxClusterSplits && attn_tc_available())
+    return launch_attn_tc(p, *desc, static_cast<cudaStream_t>(stream));
+
   dim3 grid(splits, desc->H, desc->B);
   if (cluster) {
     cudaLaunchConfig_t cfg = {};

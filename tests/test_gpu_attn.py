@@ -12,6 +12,18 @@ from util import (ATTN_MAX_ABS, ATTN_MEAN_ABS, assert_attn_close, bits_to_torch,
 
 pytestmark = pytest.mark.gpu
 
+# Every test in this file runs twice: on the default (tcgen05) kernel and on the legacy
+# mma.sync kernels selected through the descriptor flag.
+ATTN_FLAGS = 0
+
+
+@pytest.fixture(autouse=True, params=[0, sv.ATTN_FLAG_LEGACY_MMA], ids=["tcgen05", "legacy_mma"])
+def _attn_path(request):
+    global ATTN_FLAGS
+    ATTN_FLAGS = request.param
+    yield
+    ATTN_FLAGS = 0
+
 
 def run_attn(q_bits, k_bits, v_bits, prefix_len, masks=None, parents=None, num_splits=0, scale=0.0,
              out_fill=None):
@@ -26,13 +38,13 @@ def run_attn(q_bits, k_bits, v_bits, prefix_len, masks=None, parents=None, num_s
     mk = mask_to_torch(np.asarray(masks)) if masks is not None else None
     par = torch.tensor(np.asarray(parents), dtype=torch.int32, device="cuda") if parents is not None else None
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    desc = sv.make_attn_desc(q, k, v, out, num_splits, scale)
+    desc = sv.make_attn_desc(q, k, v, out, num_splits, scale, ATTN_FLAGS)
     ws = sv.alloc_attn_workspace(desc, q.device)
     sv.specvlm_tree_verify_attn(q, k, v, pl, par, mk, out, workspace=ws, status=status, desc=desc)
     torch.cuda.synchronize()
     # the workspace must be left ready for the next call: run again and compare bytes
     out2 = torch.empty_like(q)
-    desc2 = sv.make_attn_desc(q, k, v, out2, num_splits, scale)
+    desc2 = sv.make_attn_desc(q, k, v, out2, num_splits, scale, ATTN_FLAGS)
     sv.specvlm_tree_verify_attn(q, k, v, pl, par, mk, out2, workspace=ws, status=status, desc=desc2)
     torch.cuda.synchronize()
     a, b = torch_to_bits(out), torch_to_bits(out2)
@@ -225,7 +237,7 @@ def test_strided_token_major_layout_and_custom_scale():
     out = out_store.permute(0, 2, 1, 3)
     pl = torch.tensor([P, P - 37], dtype=torch.int32, device="cuda")
     mk = mask_to_torch(np.array([mask, mask]))
-    desc = sv.make_attn_desc(qt, kt, vt, out, 3, scale)
+    desc = sv.make_attn_desc(qt, kt, vt, out, 3, scale, ATTN_FLAGS)
     ws = sv.alloc_attn_workspace(desc, qt.device)
     sv.specvlm_tree_verify_attn(qt, kt, vt, pl, None, mk, out, workspace=ws, desc=desc)
     torch.cuda.synchronize()
@@ -256,7 +268,7 @@ def test_output_rows_beyond_tree_and_neighbours_untouched():
     store = torch.full((B, H, T + 6, D), 7.0, dtype=torch.bfloat16, device="cuda")
     out = store[:, :, 3:3 + T, :]
     pl = torch.tensor([P], dtype=torch.int32, device="cuda")
-    desc = sv.make_attn_desc(q, k, v, out, 2, 0.0)
+    desc = sv.make_attn_desc(q, k, v, out, 2, 0.0, ATTN_FLAGS)
     ws = sv.alloc_attn_workspace(desc, q.device)
     sv.specvlm_tree_verify_attn(q, k, v, pl, None, mask_to_torch(np.array([mask])), out, workspace=ws, desc=desc)
     torch.cuda.synchronize()
