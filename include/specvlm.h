@@ -62,8 +62,22 @@ extern "C" {
 #define SPECVLM_STATUS_BAD_ACCEPT 4  /* accept_len / accepted_idx out of range         */
 #define SPECVLM_STATUS_TIMEOUT 8     /* a bounded on-chip wait gave up                  */
 
-/* specvlm_attn_desc.flags: run the older mma.sync kernels instead of the tcgen05 kernel */
+/* specvlm_attn_desc.flags */
+/* run the older mma.sync kernels instead of the tcgen05 kernel */
 #define SPECVLM_ATTN_FLAG_LEGACY_MMA 1
+/* The attention kernel is launched so that it may start while the kernel enqueued before it
+ * on the same stream is still draining (programmatic dependent launch). By default it reads
+ * nothing until that kernel has completed. The two flags below are promises by the caller
+ * that let it start reading earlier:
+ * PREFIX_STABLE: prefix_len and the cache slots below prefix_len[b] are not written by that
+ *   preceding kernel (true in a decoder layer, where the preceding kernel produces only q and
+ *   the tree's own K/V rows): prefix tiles are prefetched early; q, the tree arrays and the
+ *   tree slots are read only after the preceding kernel has completed.
+ * INPUTS_STABLE: nothing this call reads is written by the preceding kernel, and `out` is
+ *   neither read nor written by it: the whole call may overlap with it (back-to-back
+ *   attention calls on independent inputs, as in a benchmark). */
+#define SPECVLM_ATTN_FLAG_PREFIX_STABLE 2
+#define SPECVLM_ATTN_FLAG_INPUTS_STABLE 4
 
 #define SPECVLM_MAX_TREE 64
 #define SPECVLM_HEAD_DIM 128

@@ -136,6 +136,8 @@ def specvlm_version() -> int:
 
 
 ATTN_FLAG_LEGACY_MMA = 1
+ATTN_FLAG_PREFIX_STABLE = 2
+ATTN_FLAG_INPUTS_STABLE = 4
 
 
 def make_attn_desc(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,

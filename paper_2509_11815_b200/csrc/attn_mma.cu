@@ -426,14 +426,17 @@ int resolve_num_splits(const specvlm_attn_desc& d) {
       const int64_t target = 2 * static_cast<int64_t>(sm_count());
       splits = static_cast<int>((target + bh - 1) / bh);
       if (splits > kMaxClusterSplits && splits <= 2 * kMaxClusterSplits) splits = kMaxClusterSplits;
+    } else if (d.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) {
+      // launches overlap one another: few CTAs per launch, little or no split exchange
+      splits = static_cast<int>((32 + bh - 1) / bh);
+      if (splits > kMaxClusterSplits) splits = kMaxClusterSplits;
     } else {
       // one CTA per SM, the splits of a (sequence, head) in one cluster
       splits = static_cast<int>(sm_count() / bh);
       if (splits > kMaxClusterSplits) splits = kMaxClusterSplits;
     }
   }
-  const bool tc_path = !legacy && splits <= kMaxClusterSplits;
-  const int tile = tc_path ? 128 : kTileN;
+  const int tile = (!legacy && splits <= kMaxClusterSplits) ? attn_tc_tile(d) : kTileN;
   const int max_tiles = (d.S_cap + tile - 1) / tile;
   if (splits > max_tiles) splits = max_tiles;
   if (splits > 64) splits = 64;
@@ -508,6 +511,7 @@ extern "C" int specvlm_tree_verify_attn(const uint16_t* q, const uint16_t* k_cac
   p.part_ml = workspace ? reinterpret_cast<float*>(static_cast<char*>(workspace) + counters_bytes(*desc)) : nullptr;
   p.part_o = workspace ? p.part_ml + bh * splits * kRows * 2 : nullptr;
   p.B = desc->B; p.H = desc->H; p.T = desc->T; p.S_cap = desc->S_cap; p.splits = splits;
+  p.flags = desc->flags;
   const float scale = desc->softmax_scale > 0.f ? desc->softmax_scale : 1.0f / sqrtf(static_cast<float>(kD));
   p.scale_log2 = scale * 1.4426950408889634f;
   p.q_sb = desc->q_stride_b; p.q_sh = desc->q_stride_h; p.q_st = desc->q_stride_t;
@@ -638,6 +642,7 @@ extern "C" int specvlm_tree_verify_attn_static(const uint16_t* q, const uint16_t
   p.part_ml = reinterpret_cast<float*>(scratch + kStaticCounterBytes);
   p.part_o = reinterpret_cast<float*>(scratch + kStaticCounterBytes + kStaticMlBytes);
   p.B = desc->B; p.H = desc->H; p.T = desc->T; p.S_cap = desc->S_cap; p.splits = splits;
+  p.flags = desc->flags;
   const float scale = desc->softmax_scale > 0.f ? desc->softmax_scale : 1.0f / sqrtf(static_cast<float>(kD));
   p.scale_log2 = scale * 1.4426950408889634f;
   p.q_sb = desc->q_stride_b; p.q_sh = desc->q_stride_h; p.q_st = desc->q_stride_t;

@@ -1,25 +1,28 @@
 // Tree-verification attention on the Blackwell tensor path (sm_100a): tcgen05.mma with TMEM
-// accumulators, TMA-staged K/V tiles, warp-specialised roles, cluster/DSMEM split combine.
+// accumulators, TMA-staged K/V tiles, warp-specialised roles, cluster/DSMEM split combine,
+// programmatic dependent launch.
 //
-// What it computes is the same as the legacy kernel: tree attention of the <= 64 draft-tree
-// queries over the KV prefix plus the tree's own slots (Sections 3.1, 4.1), streaming the KV
-// cache once from HBM (Section 3.2).
+// What it computes: tree attention of the <= 64 draft-tree queries over the KV prefix plus the
+// tree's own slots (Sections 3.1, 4.1), streaming the KV cache once from HBM (Section 3.2).
 //
 // One CTA per (sequence, head, split); the splits of one (sequence, head) are one thread-block
-// cluster. Roles inside a CTA (192 threads):
-//   warp 0      TMA producer: Q once, then 128-key K and V tiles into a 3-stage ring
-//               (cp.async.bulk.tensor, 128-byte swizzle, no multicast); owns the TMEM allocation
-//   warp 1      one lane issues tcgen05.mma: S = Q K^T (M=64, N=128, K=16 x 8) into one of two
-//               TMEM buffers, O += P V (M=64, N=128, K=16 x 8); tcgen05.commit signals mbarriers
-//   warps 2..5  softmax: tcgen05.ld of their 16 rows of S, scale, tree mask (one 64-bit word per
-//               row, applied with selects), running max with a lazy rescale of O in TMEM, exp2,
-//               bf16 P written to shared memory in the K-major swizzled operand layout
-// Key tiles are anchored at the END of the sequence (tile j covers keys
-// [n - 128 (j+1), n - 128 j)): the tree slots always fall in the last tile, the first tile may
-// start at a negative key index, which TMA fills with zeros, and no tile ever contains a cache
-// slot beyond prefix + T, so uninitialised slots are never loaded.
-// Every mbarrier wait is bounded; a wait that gives up sets SPECVLM_STATUS_TIMEOUT, the CTA
-// still reaches the cluster barriers, frees its TMEM and returns.
+// cluster. A CTA uses less than half of an SM (about 105 KB of shared memory, 256 TMEM columns),
+// so the CTAs of the next launch can become resident while this launch drains.
+// Roles inside a CTA (192 threads):
+//   warp 0      TMA producer: Q once, then 64-key K tiles (ring of 3) and V tiles (ring of 2)
+//               with cp.async.bulk.tensor, 128-byte swizzle, no multicast; owns the TMEM allocation
+//   warp 1      one lane issues tcgen05.mma: S = Q K^T (M=64, N=64, K=16 x 8) into one of two TMEM
+//               buffers, O += P V (M=64, N=128, K=16 x 4); tcgen05.commit signals the mbarriers
+//   warps 2..5  softmax: tcgen05.ld of their 16 rows of S, tree mask as one 64-bit visibility word
+//               per row and tile, running max with a lazy rescale of O in TMEM, exp2, bf16 P
+//               written to shared memory in the K-major swizzled operand layout
+// Key tiles are anchored at the END of the sequence (tile j covers keys [n - 64 (j+1), n - 64 j)),
+// so the tree slots always fall in tile 0, the lowest tile may start at a negative key index,
+// which TMA fills with zeros, and no tile contains a cache slot beyond prefix + T: uninitialised
+// slots are never loaded. A CTA walks its tiles from low keys to high keys, so the tile with the
+// tree slots comes last.
+// Every mbarrier wait is bounded; a wait that gives up sets SPECVLM_STATUS_TIMEOUT, the CTA still
+// reaches the cluster barriers, frees its TMEM and returns.
 #include "attn_params.cuh"
 
 #include <cooperative_groups.h>
@@ -35,36 +38,49 @@ namespace tc {
 
 constexpr int kD = SPECVLM_HEAD_DIM;
 constexpr int kRows = 64;      // MMA M: padded tree queries
-constexpr int kTile = 128;     // keys per tile
-constexpr int kStages = 3;
 constexpr int kThreads = 192;
 constexpr int kSoftmaxWarp0 = 2;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units; P stays <= 2^8
+constexpr int kLandStride = kD + 4;        // floats per exchange row: 128 values, (max, sum), padding
 
-// shared memory map (offsets from a 1024-byte aligned base)
-constexpr int kQBytes = kRows * kD * 2;        // 16 KB: two 64x64 swizzle atoms
-constexpr int kPBytes = kRows * kTile * 2;     // 16 KB: two 64x64 swizzle atoms
-constexpr int kKBytes = kTile * kD * 2;        // 32 KB: two 128x64 boxes
-constexpr int kVBytes = kTile * kD * 2;        // 32 KB
-constexpr int kStageBytes = kKBytes + kVBytes;
-constexpr int kOffQ = 0;
-constexpr int kOffP = kOffQ + kQBytes;
-constexpr int kOffStage = kOffP + kPBytes;
-constexpr int kOffBar = kOffStage + kStages * kStageBytes;
-constexpr int kNumBars = 3 * kStages + 2 + 2 + 1 + 1 + 1;
-constexpr int kOffMisc = kOffBar + kNumBars * 8;
-constexpr int kSmemBytes = kOffMisc + 64 + 1024;  // + alignment slack
-static_assert(kSmemBytes <= 232448, "shared memory budget");
+// Two configurations of the same kernel:
+//   throughput: 64-key tiles, K ring 3 / V ring 2, half an SM per CTA (two CTAs per SM, so the next
+//               launch can become resident while this one drains)
+//   latency   : 128-key tiles, K ring 3 / V ring 3, a whole SM per CTA (deepest prefetch for one launch)
+template <int TILE_, int KS_, int VS_, int MINB_>
+struct Cfg {
+  static constexpr int kTile = TILE_;         // keys per tile
+  static constexpr int kKStages = KS_;
+  static constexpr int kVStages = VS_;
+  static constexpr int kMinBlocks = MINB_;
+  static constexpr int kHalves = TILE_ / 64;  // 64-key swizzle atoms per tile
+  // shared memory map (offsets from a 1024-byte aligned base)
+  static constexpr int kQBytes = kRows * kD * 2;      // two 64x64 swizzle atoms (d halves)
+  static constexpr int kPBytes = kRows * TILE_ * 2;   // kHalves 64x64 swizzle atoms
+  static constexpr int kKBytes = TILE_ * kD * 2;      // two TILE-row x 128-byte boxes (d halves)
+  static constexpr int kVBytes = TILE_ * kD * 2;
+  static constexpr int kOffQ = 0;
+  static constexpr int kOffP = kOffQ + kQBytes;
+  static constexpr int kOffK = kOffP + kPBytes;
+  static constexpr int kOffV = kOffK + KS_ * kKBytes;
+  static constexpr int kOffBar = kOffV + VS_ * kVBytes;
+  static constexpr int kNumBars = 2 * KS_ + 2 * VS_ + 2 + 2 + 1 + 1 + 1 + 1;
+  static constexpr int kOffMisc = kOffBar + kNumBars * 8;
+  static constexpr int kSmemBytes = kOffMisc + 64 + 1024;  // + alignment slack
+  static_assert(kSmemBytes <= (MINB_ == 2 ? 115712 : 232448), "shared memory budget");
+  // staging + landing zones of the split exchange: 2 * ns * ceil(64/ns) rows (worst case ns = 7)
+  static_assert(2 * 7 * 10 * kLandStride * 4 <= KS_ * kKBytes + VS_ * kVBytes, "exchange zones");
+  // TMEM columns: S0 [0,TILE), S1 [TILE,2 TILE), O [2 TILE, 2 TILE + 128)
+  static constexpr uint32_t kTmemCols = TILE_ == 64 ? 256 : 512;
+  static constexpr uint32_t kColS0 = 0, kColS1 = TILE_, kColO = 2 * TILE_;
+};
+using CfgThroughput = Cfg<64, 3, 2, 2>;
+using CfgLatency = Cfg<128, 3, 3, 1>;
 
-// TMEM columns: S0 [0,128), S1 [128,256), O [256,384); 512 allocated (power of two)
-constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256;
-
-// tcgen05 instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M=64, N=128
-constexpr uint32_t make_idesc(bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | ((b_mn_major ? 1u : 0u) << 16) |
-         ((128u >> 3) << 17) | ((64u >> 4) << 24);
+// tcgen05 instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, K-major A, M = 64
+constexpr uint32_t make_idesc(uint32_t n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((64u >> 4) << 24);
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -89,7 +105,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false after kSpinLimit unsuccessful polls or once another role has given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 1023u) == 1023u && *abort_flag) return false;
@@ -106,6 +122,10 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
+
+// ---- programmatic dependent launch
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ---- tcgen05
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -144,39 +164,67 @@ __device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&r)[32]) {
         "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
       : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_st64(uint32_t taddr, const float (&r)[32]) {
+// 16 lanes x 32 columns: r[4j+e], j = 0..3
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[16]) {
+  uint32_t* u = reinterpret_cast<uint32_t*>(r);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+        "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&r)[16]) {
   const uint32_t* u = reinterpret_cast<const uint32_t*>(r);
   asm volatile(
-      "tcgen05.st.sync.aligned.16x256b.x8.b32 [%32], "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
+      "tcgen05.st.sync.aligned.16x256b.x4.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
       ::"r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7]),
         "r"(u[8]), "r"(u[9]), "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15]),
-        "r"(u[16]), "r"(u[17]), "r"(u[18]), "r"(u[19]), "r"(u[20]), "r"(u[21]), "r"(u[22]), "r"(u[23]),
-        "r"(u[24]), "r"(u[25]), "r"(u[26]), "r"(u[27]), "r"(u[28]), "r"(u[29]), "r"(u[30]), "r"(u[31]),
         "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// 2^x; -inf -> 0
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
-struct Barriers {
-  uint32_t full_k[kStages], full_v[kStages], empty[kStages];
-  uint32_t s_full[2], s_free[2];
-  uint32_t p_full, pv_done, q_full;
-};
+// Address of the same shared-memory offset in the CTA of rank `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, int rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_f32x2(uint32_t addr, float a, float b) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
+
+#ifdef SPECVLM_TC_TRACE
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define TRACE(slot) do { if (trace_on) trace[(slot)] = gtime(); } while (0)
+#else
+#define TRACE(slot) do { } while (0)
+#endif
 
 }  // namespace tc
 
 using namespace tc;
 
-__global__ void __launch_bounds__(kThreads, 1)
+template <class C>
+__global__ void __launch_bounds__(kThreads, C::kMinBlocks)
 tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_q,
                     const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
+  constexpr int kTile = C::kTile, kKStages = C::kKStages, kVStages = C::kVStages, kHalves = C::kHalves;
+  constexpr int kQBytes = C::kQBytes, kKBytes = C::kKBytes, kVBytes = C::kVBytes;
+  constexpr int kOffQ = C::kOffQ, kOffP = C::kOffP, kOffK = C::kOffK, kOffV = C::kOffV, kOffBar = C::kOffBar;
+  constexpr int kNumBars = C::kNumBars, kOffMisc = C::kOffMisc;
+  constexpr uint32_t kTmemCols = C::kTmemCols, kColS0 = C::kColS0, kColS1 = C::kColS1, kColO = C::kColO;
   extern __shared__ unsigned char smem_raw[];
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
@@ -188,48 +236,37 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int T = p.T;
+#ifdef SPECVLM_TC_TRACE
+  long long* trace = reinterpret_cast<long long*>(p.counters) + 64 * (blockIdx.y * gridDim.x + blockIdx.x);
+  const bool trace_on = p.counters != nullptr && lane == 0 && blockIdx.z == 0;
+  if (warp <= 2) TRACE(warp);
+#endif
 
-  Barriers bar;
-  {
-    uint32_t a = base + kOffBar;
-    for (int s = 0; s < kStages; ++s) { bar.full_k[s] = a; a += 8; }
-    for (int s = 0; s < kStages; ++s) { bar.full_v[s] = a; a += 8; }
-    for (int s = 0; s < kStages; ++s) { bar.empty[s] = a; a += 8; }
-    bar.s_full[0] = a; a += 8; bar.s_full[1] = a; a += 8;
-    bar.s_free[0] = a; a += 8; bar.s_free[1] = a; a += 8;
-    bar.p_full = a; a += 8; bar.pv_done = a; a += 8; bar.q_full = a; a += 8;
-  }
+  // barrier addresses: full_k[] empty_k[] full_v[] empty_v[] s_full[2] s_free[2] p_full pv_done q_full land_full
+  const uint32_t bar0 = base + kOffBar;
+  auto FULL_K = [&](int s) { return bar0 + 8u * s; };
+  auto EMPTY_K = [&](int s) { return bar0 + 8u * (kKStages + s); };
+  auto FULL_V = [&](int s) { return bar0 + 8u * (2 * kKStages + s); };
+  auto EMPTY_V = [&](int s) { return bar0 + 8u * (2 * kKStages + kVStages + s); };
+  const uint32_t bar1 = bar0 + 8u * (2 * kKStages + 2 * kVStages);
+  auto S_FULL = [&](int i) { return bar1 + 8u * i; };
+  auto S_FREE = [&](int i) { return bar1 + 8u * (2 + i); };
+  const uint32_t P_FULL = bar1 + 32, PV_DONE = bar1 + 40, Q_FULL = bar1 + 48, LAND_FULL = bar1 + 56;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 8);
 
-  // ---- sequence geometry (tiles are anchored at the end of the sequence)
-  int P = p.prefix_len[b];
-  int n_keys = P + T;
-  if (P < 0 || n_keys > p.S_cap) {
-    if (threadIdx.x == 0 && split == 0 && h == 0 && p.status != nullptr)
-      atomicOr(p.status, SPECVLM_STATUS_BAD_PREFIX);
-    P = 0;
-    n_keys = 0;
-  }
-  const int tiles_total = (n_keys + kTile - 1) / kTile;
-  const int tps = (tiles_total + p.splits - 1) / p.splits;
-  const int tile_begin = min(split * tps, tiles_total);  // tile index counted from the end
-  const int n_tiles = min(tile_begin + tps, tiles_total) - tile_begin;
+  const bool inputs_stable = (p.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) != 0;
+  const bool prefix_stable = inputs_stable || (p.flags & SPECVLM_ATTN_FLAG_PREFIX_STABLE) != 0;
 
-  // ---- set-up: barriers, TMEM
+  // ---- set-up that touches no global input: tensor-map prefetch, barriers, TMEM
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar.full_k[s], 1);
-      mbar_init(bar.full_v[s], 1);
-      mbar_init(bar.empty[s], 1);
-    }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar.s_full[i], 1);
-      mbar_init(bar.s_free[i], 128);
-    }
-    mbar_init(bar.p_full, 128);
-    mbar_init(bar.pv_done, 1);
-    mbar_init(bar.q_full, 1);
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
+    for (int i = 0; i < kNumBars; ++i) mbar_init(bar0 + 8u * i, 1);
+    mbar_init(S_FREE(0), 128);
+    mbar_init(S_FREE(1), 128);
+    mbar_init(P_FULL, 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -239,108 +276,177 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
                  "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // The next launch on the stream may begin its own set-up now; it decides itself what it may read.
+  pdl_launch_dependents();
+  if (!prefix_stable) pdl_wait();  // everything below reads memory the preceding kernel may have written
+  const int prefix_raw = p.prefix_len[b];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+#ifdef SPECVLM_TC_TRACE
+  if (warp <= 2) TRACE(3 + warp);
+#endif
 
-  // softmax-warp state that outlives the main loop
-  float o[16][4];
-  float mu0 = -INFINITY, mu1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-  const int sw = warp - kSoftmaxWarp0;       // 0..3 for softmax warps
-  const int quad = warp & 3;                 // TMEM lane quadrant this warp may access
+  // ---- sequence geometry
+  int P = prefix_raw;
+  int n_keys = P + T;
+  if (P < 0 || n_keys > p.S_cap) {
+    if (threadIdx.x == 0 && split == 0 && h == 0 && p.status != nullptr)
+      atomicOr(p.status, SPECVLM_STATUS_BAD_PREFIX);
+    P = 0;
+    n_keys = 0;
+  }
+  const int tiles_total = (n_keys + kTile - 1) / kTile;
+  const int tps = (tiles_total + p.splits - 1) / p.splits;
+  const int tile_begin = min(split * tps, tiles_total);  // tile index counted from the end of the sequence
+  const int n_tiles = min(tile_begin + tps, tiles_total) - tile_begin;
+  // step i of this CTA works on tile (tile_begin + n_tiles - 1 - i): low keys first, tree slots last
+  auto KEY0 = [&](int i) { return n_keys - (tile_begin + n_tiles - i) * kTile; };
+
+  const int sw = warp - kSoftmaxWarp0;  // 0..3 for softmax warps
+  const int quad = warp & 3;            // TMEM lane quadrant this warp may access
   const int g = lane >> 2, t4 = lane & 3;
   const int row0 = quad * 16 + g, row1 = row0 + 8;
+  const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
+  float mu0 = -INFINITY, mu1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
   if (warp == 0) {
     // ======================= TMA producer =======================
+    // K and V rings advance independently: a slot is refilled as soon as the MMAs that read it
+    // have completed, whichever ring that is.
     if (lane == 0 && n_tiles > 0) {
-      mbar_expect_tx(bar.q_full, kQBytes);
-      tma_load_4d(base + kOffQ, &map_q, bar.q_full, 0, 0, h, b);
-      tma_load_4d(base + kOffQ + kQBytes / 2, &map_q, bar.q_full, 64, 0, h, b);
-      int issued = 0;
-      for (int i = 0; i < n_tiles; ++i) {
-        const int s = i % kStages;
-        if (i >= kStages && !mbar_wait(bar.empty[s], ((i / kStages) & 1) ^ 1, abort_flag)) break;
-        const int key0 = n_keys - (tile_begin + i + 1) * kTile;  // may be negative: zero-filled
-        const uint32_t sk = base + kOffStage + s * kStageBytes, sv = sk + kKBytes;
-        mbar_expect_tx(bar.full_k[s], kKBytes);
-        tma_load_4d(sk, &map_k, bar.full_k[s], 0, key0, h, b);
-        tma_load_4d(sk + kKBytes / 2, &map_k, bar.full_k[s], 64, key0, h, b);
-        mbar_expect_tx(bar.full_v[s], kVBytes);
-        tma_load_4d(sv, &map_v, bar.full_v[s], 0, key0, h, b);
-        tma_load_4d(sv + kVBytes / 2, &map_v, bar.full_v[s], 64, key0, h, b);
-        ++issued;
+      auto issue_q = [&]() {
+        mbar_expect_tx(Q_FULL, kQBytes);
+        tma_load_4d(base + kOffQ, &map_q, Q_FULL, 0, 0, h, b);
+        tma_load_4d(base + kOffQ + kQBytes / 2, &map_q, Q_FULL, 64, 0, h, b);
+      };
+      auto issue_k = [&](int i) {
+        const int sk = i % kKStages;
+        const uint32_t dk = base + kOffK + sk * kKBytes;
+        mbar_expect_tx(FULL_K(sk), kKBytes);
+        tma_load_4d(dk, &map_k, FULL_K(sk), 0, KEY0(i), h, b);
+        tma_load_4d(dk + kKBytes / 2, &map_k, FULL_K(sk), 64, KEY0(i), h, b);
+      };
+      auto issue_v = [&](int i) {
+        const int sv = i % kVStages;
+        const uint32_t dv = base + kOffV + sv * kVBytes;
+        mbar_expect_tx(FULL_V(sv), kVBytes);
+        tma_load_4d(dv, &map_v, FULL_V(sv), 0, KEY0(i), h, b);
+        tma_load_4d(dv + kVBytes / 2, &map_v, FULL_V(sv), 64, KEY0(i), h, b);
+        TRACE(8 + (i < 12 ? i : 12));
+      };
+      int ik = 0, iv = 0;
+      if (prefix_stable && !inputs_stable) {
+        // Pure prefix tiles may be fetched before the preceding kernel has completed; Q, the tree
+        // arrays and the tile with the tree slots are read only afterwards.
+        while (ik < n_tiles && ik < kKStages && KEY0(ik) + kTile <= P) issue_k(ik++);
+        while (iv < n_tiles && iv < kVStages && KEY0(iv) + kTile <= P) issue_v(iv++);
+        pdl_wait();
+      }
+      issue_q();
+      uint32_t idle = 0;
+      while (ik < n_tiles || iv < n_tiles) {
+        bool progress = false;
+        if (ik < n_tiles && (ik < kKStages || mbar_try_wait(EMPTY_K(ik % kKStages), ((ik / kKStages) & 1) ^ 1))) {
+          issue_k(ik++);
+          progress = true;
+        }
+        if (iv < n_tiles && (iv < kVStages || mbar_try_wait(EMPTY_V(iv % kVStages), ((iv / kVStages) & 1) ^ 1))) {
+          issue_v(iv++);
+          progress = true;
+        }
+        if (progress) {
+          idle = 0;
+        } else if (++idle > kSpinLimit || ((idle & 1023u) == 0 && *abort_flag)) {
+          *abort_flag = 1;
+          break;
+        }
       }
       if (*abort_flag) {
         // give copies that are still in flight a bounded time to land before the CTA exits
-        mbar_wait(bar.q_full, 0, abort_flag);
-        for (int i = max(0, issued - kStages); i < issued; ++i) {
+        for (int i = max(0, ik - kKStages); i < ik; ++i) {
           uint32_t spins = 0;
-          while (!mbar_try_wait(bar.full_k[i % kStages], (i / kStages) & 1) && ++spins < kSpinLimit) {}
-          spins = 0;
-          while (!mbar_try_wait(bar.full_v[i % kStages], (i / kStages) & 1) && ++spins < kSpinLimit) {}
+          while (!mbar_try_wait(FULL_K(i % kKStages), (i / kKStages) & 1) && ++spins < kSpinLimit) {}
+        }
+        for (int i = max(0, iv - kVStages); i < iv; ++i) {
+          uint32_t spins = 0;
+          while (!mbar_try_wait(FULL_V(i % kVStages), (i / kVStages) & 1) && ++spins < kSpinLimit) {}
         }
       }
     }
   } else if (warp == 1) {
     // ======================= MMA issuer =======================
     if (lane == 0 && n_tiles > 0) {
-      constexpr uint32_t idesc_qk = make_idesc(false), idesc_pv = make_idesc(true);
+      constexpr uint32_t idesc_qk = make_idesc(kTile, false), idesc_pv = make_idesc(kD, true);
       const uint32_t tmem_o = tmem_base + kColO;
-      bool ok = mbar_wait(bar.q_full, 0, abort_flag);
       auto issue_qk = [&](int i) {
-        const int s = i % kStages;
-        const uint32_t sk = base + kOffStage + s * kStageBytes;
+        const int sk = i % kKStages;
+        const uint32_t ak = base + kOffK + sk * kKBytes;
         const uint32_t tmem_s = tmem_base + ((i & 1) ? kColS1 : kColS0);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
           const uint64_t ad = make_desc(base + kOffQ + (ks >> 2) * (kQBytes / 2) + (ks & 3) * 32, 16, 1024);
-          const uint64_t bd = make_desc(sk + (ks >> 2) * (kKBytes / 2) + (ks & 3) * 32, 16, 1024);
+          const uint64_t bd = make_desc(ak + (ks >> 2) * (kKBytes / 2) + (ks & 3) * 32, 16, 1024);
           tc_mma(tmem_s, ad, bd, idesc_qk, ks > 0 ? 1u : 0u);
         }
-        tc_commit(bar.s_full[i & 1]);
+        tc_commit(EMPTY_K(sk));  // K stage free once these MMAs have read it
+        tc_commit(S_FULL(i & 1));
       };
-      if (ok) ok = mbar_wait(bar.full_k[0], 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        issue_qk(0);
-      }
-      for (int i = 0; ok && i < n_tiles; ++i) {
-        const int s = i % kStages;
-        if (i + 1 < n_tiles) {
-          const int s1 = (i + 1) % kStages;
-          ok = mbar_wait(bar.full_k[s1], ((i + 1) / kStages) & 1, abort_flag);
-          if (ok && i + 1 >= 2) ok = mbar_wait(bar.s_free[(i + 1) & 1], (((i + 1) >> 1) & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          issue_qk(i + 1);
-        }
-        ok = mbar_wait(bar.full_v[s], (i / kStages) & 1, abort_flag);
-        if (ok) ok = mbar_wait(bar.p_full, i & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t sv = base + kOffStage + s * kStageBytes + kKBytes;
+      auto issue_pv = [&](int i) {
+        const int sv = i % kVStages;
+        const uint32_t av = base + kOffV + sv * kVBytes;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint64_t ad = make_desc(base + kOffP + (ks >> 2) * (kPBytes / 2) + (ks & 3) * 32, 16, 1024);
-          const uint64_t bd = make_desc(sv + ks * 2048, kVBytes / 2, 1024);
+        for (int ks = 0; ks < kTile / 16; ++ks) {
+          const uint64_t ad = make_desc(base + kOffP + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
+          const uint64_t bd = make_desc(av + ks * 2048, kVBytes / 2, 1024);
           tc_mma(tmem_o, ad, bd, idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
         }
-        tc_commit(bar.empty[s]);
-        tc_commit(bar.pv_done);
+        tc_commit(EMPTY_V(sv));
+        tc_commit(PV_DONE);
+      };
+      // Whichever of "O += P V of tile ip" and "S = Q K^T of tile iq" has its operands ready is
+      // issued; PV is looked at first because the softmax warps wait for its completion.
+      bool ok = mbar_wait(Q_FULL, 0, abort_flag);
+      int iq = 0, ip = 0;
+      uint32_t idle = 0;
+      while (ok && ip < n_tiles) {
+        bool progress = false;
+        if (ip < iq && mbar_try_wait(P_FULL, ip & 1) && mbar_try_wait(FULL_V(ip % kVStages), (ip / kVStages) & 1)) {
+          tc_fence_after();
+#ifdef SPECVLM_TC_TRACE
+          if (ip < 8) TRACE(47 + 2 * ip);
+#endif
+          issue_pv(ip++);
+          progress = true;
+        }
+        if (iq < n_tiles && iq < ip + 2 && mbar_try_wait(FULL_K(iq % kKStages), (iq / kKStages) & 1) &&
+            (iq < 2 || mbar_try_wait(S_FREE(iq & 1), ((iq >> 1) & 1) ^ 1))) {
+          tc_fence_after();
+#ifdef SPECVLM_TC_TRACE
+          if (iq < 8) TRACE(48 + 2 * iq);
+#endif
+          issue_qk(iq++);
+          progress = true;
+        }
+        if (progress) {
+          idle = 0;
+        } else if (++idle > kSpinLimit || ((idle & 1023u) == 0 && *abort_flag)) {
+          *abort_flag = 1;
+          ok = false;
+        }
       }
     }
   } else {
     // ======================= softmax warps =======================
+    if (prefix_stable && !inputs_stable) pdl_wait();  // the tree arrays may come from the preceding kernel
     uint64_t mask0 = 0, mask1 = 0;
     if (p.mask != nullptr) {
       if (row0 < T) mask0 = p.mask[b * T + row0];
       if (row1 < T) mask1 = p.mask[b * T + row1];
     } else {
       const int32_t* par = p.parent + b * T;
+#pragma unroll 1
       for (int pass = 0; pass < 2; ++pass) {
         const int row = pass ? row1 : row0;
         uint64_t bits = 0;
@@ -355,38 +461,55 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
         if (pass) mask1 = bits; else mask0 = bits;
       }
     }
-    const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
+    const uint64_t tmask = (T >= 64) ? ~0ull : ((1ull << T) - 1ull);
+    mask0 &= tmask;
+    mask1 &= tmask;
+    unsigned char* prow0 = smem + kOffP + row0 * 128 + t4 * 4;
+    unsigned char* prow1 = prow0 + 8 * 128;
     bool ok = true;
+#pragma unroll 1
     for (int i = 0; i < n_tiles && ok; ++i) {
-      const int key0 = n_keys - (tile_begin + i + 1) * kTile;
-      ok = mbar_wait(bar.s_full[i & 1], (i >> 1) & 1, abort_flag);
+      const int key0 = KEY0(i);
+      // visibility of the tile's columns (bit c of half hf <-> key key0 + 64 hf + c), shifted to this
+      // thread's column pair: columns [a, d) are prefix keys, column d + t is tree slot t
+      uint64_t vis0[kHalves], vis1[kHalves];
+      {
+        const int a = key0 < 0 ? -key0 : 0;
+        const int d = P - key0;
+#pragma unroll
+        for (int hf = 0; hf < kHalves; ++hf) {
+          const int lo = max(a - 64 * hf, 0), hi = min(d - 64 * hf, 64);
+          uint64_t pre = 0;
+          if (hi > lo) pre = ((~0ull) >> (64 - (hi - lo))) << lo;
+          const int sh = d - 64 * hf;  // column of tree slot 0 in this half
+          uint64_t t0 = 0, t1 = 0;
+          if (sh >= 0 && sh < 64) { t0 = mask0 << sh; t1 = mask1 << sh; }
+          else if (sh < 0 && sh > -64) { t0 = mask0 >> (-sh); t1 = mask1 >> (-sh); }
+          vis0[hf] = (pre | t0) >> (2 * t4);
+          vis1[hf] = (pre | t1) >> (2 * t4);
+        }
+      }
+
+      ok = mbar_wait(S_FULL(i & 1), (i >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      float s[2][32];
-      const uint32_t ts = tmem_base + lane_base + ((i & 1) ? kColS1 : kColS0);
-      tmem_ld64(ts, s[0]);
-      tmem_ld64(ts + 64, s[1]);
+      float s[kHalves][32];
+#pragma unroll
+      for (int hf = 0; hf < kHalves; ++hf)
+        tmem_ld64(tmem_base + lane_base + ((i & 1) ? kColS1 : kColS0) + 64 * hf, s[hf]);
       tmem_wait_ld();
       tc_fence_before();
-      mbar_arrive(bar.s_free[i & 1]);
+      mbar_arrive(S_FREE(i & 1));
 
-      // scale (log2 domain) and mask: key >= 0; prefix keys visible; tree slot t visible iff mask bit t
-      const bool need_mask = (key0 < 0) || (key0 + kTile > P);
       float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
+      for (int hf = 0; hf < kHalves; ++hf) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            float x = s[hf][4 * j + e] * p.scale_log2;
-            if (need_mask) {
-              const int key = key0 + hf * 64 + j * 8 + t4 * 2 + (e & 1);
-              const uint64_t mw = (e & 2) ? mask1 : mask0;
-              const int t = key - P;
-              const bool vis = (key >= 0) && ((t < 0) || ((mw >> (t & 63)) & 1ull));
-              x = vis ? x : -INFINITY;
-            }
+            const bool v = (((e & 2) ? vis1[hf] : vis0[hf]) >> (8 * j + (e & 1))) & 1ull;
+            const float x = v ? s[hf][4 * j + e] : -INFINITY;
             s[hf][4 * j + e] = x;
             if (e & 2) mx1 = fmaxf(mx1, x); else mx0 = fmaxf(mx0, x);
           }
@@ -396,6 +519,8 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
       mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      mx0 *= p.scale_log2;  // scores are compared and exponentiated in the log2 domain; scale > 0
+      mx1 *= p.scale_log2;
 
       // lazy rescale: the reference maximum only moves when the tile maximum exceeds it by > 2^8
       const bool need0 = (mx0 > mu0 + kRescaleThreshold) || (mu0 == -INFINITY && mx0 > -INFINITY);
@@ -404,7 +529,7 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
 
       // P is single-buffered and O is about to be touched: the previous PV must be complete
       if (i > 0) {
-        ok = mbar_wait(bar.pv_done, (i - 1) & 1, abort_flag);
+        ok = mbar_wait(PV_DONE, (i - 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
       }
@@ -414,136 +539,199 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
         if (need0) { mu0 = mx0; l0 *= a0; }
         if (need1) { mu1 = mx1; l1 *= a1; }
         if (i > 0) {
-          const uint32_t to = tmem_base + lane_base + kColO;
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            float ov[32];
-            tmem_ld64(to + hf * 64, ov);
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            const uint32_t to = tmem_base + lane_base + kColO + c * 32;
+            float ov[16];
+            tmem_ld32(to, ov);
             tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < 4; ++j) {
               ov[4 * j + 0] *= a0; ov[4 * j + 1] *= a0; ov[4 * j + 2] *= a1; ov[4 * j + 3] *= a1;
             }
-            tmem_st64(to + hf * 64, ov);
+            tmem_st32(to, ov);
           }
           tmem_wait_st();
         }
       }
-      const float ms0 = (mu0 == -INFINITY) ? 0.f : mu0;
-      const float ms1 = (mu1 == -INFINITY) ? 0.f : mu1;
+      const float nm0 = (mu0 == -INFINITY) ? 0.f : -mu0;
+      const float nm1 = (mu1 == -INFINITY) ? 0.f : -mu1;
 
       // exponentials, row sums, P as the K-major swizzled A operand: row r, key c ->
-      // atom c/64, byte r*128 + (((c%64)/8) ^ (r&7))*16 + (c%8)*2
+      // atom c/64, byte r*128 + (((c%64)/8) ^ (r&7))*16 + (c%8)*2   (r & 7 == g for both rows)
       float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
+      for (int hf = 0; hf < kHalves; ++hf) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-          const float p0 = exp2f(s[hf][4 * j + 0] - ms0), p1 = exp2f(s[hf][4 * j + 1] - ms0);
-          const float p2 = exp2f(s[hf][4 * j + 2] - ms1), p3 = exp2f(s[hf][4 * j + 3] - ms1);
+          const float p0 = ex2(fmaf(s[hf][4 * j + 0], p.scale_log2, nm0));
+          const float p1 = ex2(fmaf(s[hf][4 * j + 1], p.scale_log2, nm0));
+          const float p2 = ex2(fmaf(s[hf][4 * j + 2], p.scale_log2, nm1));
+          const float p3 = ex2(fmaf(s[hf][4 * j + 3], p.scale_log2, nm1));
           sum0 += p0 + p1;
           sum1 += p2 + p3;
-          unsigned char* atom = smem + kOffP + hf * (kPBytes / 2);
-          *reinterpret_cast<uint32_t*>(atom + row0 * 128 + ((j ^ (row0 & 7)) << 4) + t4 * 4) = pack_bf16(p0, p1);
-          *reinterpret_cast<uint32_t*>(atom + row1 * 128 + ((j ^ (row1 & 7)) << 4) + t4 * 4) = pack_bf16(p2, p3);
+          const int off = hf * 8192 + ((j ^ g) << 4);
+          *reinterpret_cast<uint32_t*>(prow0 + off) = pack_bf16(p0, p1);
+          *reinterpret_cast<uint32_t*>(prow1 + off) = pack_bf16(p2, p3);
         }
       }
       l0 += sum0;
       l1 += sum1;
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
       tc_fence_before();
-      mbar_arrive(bar.p_full);
+      mbar_arrive(P_FULL);
+#ifdef SPECVLM_TC_TRACE
+      if (warp == 2) TRACE(24 + (i < 12 ? i : 12));
+#endif
     }
-    // ---- O out of TMEM
     if (ok && n_tiles > 0) {
-      ok = mbar_wait(bar.pv_done, (n_tiles - 1) & 1, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        const uint32_t to = tmem_base + lane_base + kColO;
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          float ov[32];
-          tmem_ld64(to + hf * 64, ov);
-          tmem_wait_ld();
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            o[hf * 8 + j][0] = ov[4 * j + 0]; o[hf * 8 + j][1] = ov[4 * j + 1];
-            o[hf * 8 + j][2] = ov[4 * j + 2]; o[hf * 8 + j][3] = ov[4 * j + 3];
-          }
-        }
-      }
+      ok = mbar_wait(PV_DONE, (n_tiles - 1) & 1, abort_flag);
+      tc_fence_after();
     }
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
     l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
   }
-
-  // ---- all roles meet; from here on shared-memory stages and TMEM are no longer in use
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const bool aborted = *abort_flag != 0;
-  if (aborted && threadIdx.x == 0 && p.status != nullptr) atomicOr(p.status, SPECVLM_STATUS_TIMEOUT);
-  if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-  }
+#ifdef SPECVLM_TC_TRACE
+  if (warp <= 2) TRACE(40 + warp);
+#endif
 
   uint16_t* obase = p.out + b * p.o_sb + h * p.o_sh;
+  const bool have_o = n_tiles > 0;  // otherwise the TMEM accumulator was never written
+  const uint32_t to0 = tmem_base + lane_base + kColO;
+
   if (p.splits == 1) {
-    if (warp >= kSoftmaxWarp0 && !aborted) {
+    // ---- single split: normalise O straight out of TMEM
+    const bool aborted_local = *abort_flag != 0;
+    if (warp >= kSoftmaxWarp0 && !aborted_local) {
+      if (inputs_stable) pdl_wait();  // `out` may still be in use by the preceding kernel
       const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float ov[16];
+        if (have_o) {
+          tmem_ld32(to0 + c * 32, ov);
+          tmem_wait_ld();
+        } else {
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int col = i * 8 + t4 * 2;
-        if (row0 < T) *reinterpret_cast<uint32_t*>(obase + row0 * p.o_st + col) = pack_bf16(o[i][0] * i0, o[i][1] * i0);
-        if (row1 < T) *reinterpret_cast<uint32_t*>(obase + row1 * p.o_st + col) = pack_bf16(o[i][2] * i1, o[i][3] * i1);
+          for (int j = 0; j < 16; ++j) ov[j] = 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int col = c * 32 + j * 8 + t4 * 2;
+          if (row0 < T) *reinterpret_cast<uint32_t*>(obase + row0 * p.o_st + col) = pack_bf16(ov[4 * j] * i0, ov[4 * j + 1] * i0);
+          if (row1 < T) *reinterpret_cast<uint32_t*>(obase + row1 * p.o_st + col) = pack_bf16(ov[4 * j + 2] * i1, ov[4 * j + 3] * i1);
+        }
       }
     }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (*abort_flag != 0 && threadIdx.x == 0 && p.status != nullptr) atomicOr(p.status, SPECVLM_STATUS_TIMEOUT);
+    if (warp == 0)
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     return;
   }
 
-  // ---- partial into this CTA's shared memory, then combine across the cluster through DSMEM
-  float* so = reinterpret_cast<float*>(smem + kOffStage);  // [64][128] fp32
-  float* sml = so + kRows * kD;                            // [64][2]  (running max, running sum)
-  if (warp >= kSoftmaxWarp0) {
+  // ---- exchange through distributed shared memory. Output row r is combined by CTA r % splits.
+  // Each CTA first writes its unnormalised O rows (with the row's running max and sum in the
+  // row's padding) into a local staging area grouped by owner. After the first cluster barrier
+  // every CTA of the cluster is past its main loop, so the K/V rings are free everywhere; one
+  // thread then sends each owner its group with one bulk shared-to-shared copy that completes
+  // on the owner's mbarrier. A CTA combines its rows once its own landing zone is complete, and
+  // leaves after the second cluster barrier, when nobody can still be reading its staging area.
+  const int ns = p.splits;
+  const int rk = (kRows + ns - 1) / ns;                    // rows per (source, owner) group
+  const uint32_t group_bytes = rk * kLandStride * 4;       // multiple of 16
+  float* stage = reinterpret_cast<float*>(smem + kOffK);   // [owner][rk][kLandStride]
+  const uint32_t stage_u32 = base + kOffK;
+  const uint32_t land_u32 = stage_u32 + ns * group_bytes;  // [source][rk][kLandStride]
+  const float* landp = stage + ns * rk * kLandStride;
+  const bool aborted0 = *abort_flag != 0;
+  if (threadIdx.x == 0) mbar_expect_tx(LAND_FULL, (ns - 1) * group_bytes);  // armed before anyone may send
+  if (warp >= kSoftmaxWarp0 && !aborted0) {
+    float* d0 = stage + ((row0 % ns) * rk + row0 / ns) * kLandStride + t4 * 2;
+    float* d1 = stage + ((row1 % ns) * rk + row1 / ns) * kLandStride + t4 * 2;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      float ov[16];
+      if (have_o) {
+        tmem_ld32(to0 + c * 32, ov);
+        tmem_wait_ld();
+      } else {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      *reinterpret_cast<float2*>(so + row0 * kD + i * 8 + t4 * 2) = make_float2(o[i][0], o[i][1]);
-      *reinterpret_cast<float2*>(so + row1 * kD + i * 8 + t4 * 2) = make_float2(o[i][2], o[i][3]);
+        for (int j = 0; j < 16; ++j) ov[j] = 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        *reinterpret_cast<float2*>(d0 + c * 32 + j * 8) = make_float2(ov[4 * j + 0], ov[4 * j + 1]);
+        *reinterpret_cast<float2*>(d1 + c * 32 + j * 8) = make_float2(ov[4 * j + 2], ov[4 * j + 3]);
+      }
     }
     if (t4 == 0) {
-      *reinterpret_cast<float2*>(sml + row0 * 2) = make_float2(mu0, l0);
-      *reinterpret_cast<float2*>(sml + row1 * 2) = make_float2(mu1, l1);
+      *reinterpret_cast<float2*>(d0 + kD) = make_float2(mu0, l0);
+      *reinterpret_cast<float2*>(d1 + kD) = make_float2(mu1, l1);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // staging is read by the bulk copies
+  }
+#ifdef SPECVLM_TC_TRACE
+  if (warp == 2) TRACE(43);
+#endif
+  tc_fence_before();
+  cluster.sync();
+  tc_fence_after();
+#ifdef SPECVLM_TC_TRACE
+  if (warp == 2) TRACE(44);
+#endif
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+  if (threadIdx.x == kSoftmaxWarp0 * 32) {
+    for (int dst = 0; dst < ns; ++dst) {
+      if (dst == split) continue;
+      asm volatile(
+          "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+          ::"r"(map_to_rank(land_u32 + split * group_bytes, dst)), "r"(stage_u32 + dst * group_bytes),
+            "r"(group_bytes), "r"(map_to_rank(LAND_FULL, dst)) : "memory");
     }
   }
-  cluster.sync();
-  if (warp >= kSoftmaxWarp0 && !aborted) {
-    const int nsplit = p.splits;
-    int nth = 0;
-    for (int row = split; row < T; row += nsplit, ++nth) {
-      if ((nth & 3) != sw) continue;
-      float2 ml = make_float2(-INFINITY, 0.f);
-      if (lane < nsplit) ml = *reinterpret_cast<const float2*>(cluster.map_shared_rank(sml, lane) + row * 2);
-      float mstar = ml.x;
-#pragma unroll
-      for (int off = 4; off > 0; off >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, off));
-      const float w = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mstar);
-      float lsum = w * ml.y;
-#pragma unroll
-      for (int off = 4; off > 0; off >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, off);
-      lsum = __shfl_sync(0xffffffffu, lsum, 0);
+  bool landed = true;
+  if (warp >= kSoftmaxWarp0) landed = mbar_wait(LAND_FULL, 0, abort_flag);
+  cluster.barrier_arrive();
+#ifdef SPECVLM_TC_TRACE
+  if (warp == 2) TRACE(45);
+#endif
+  const bool aborted = *abort_flag != 0;
+  if (aborted && threadIdx.x == 0 && p.status != nullptr) atomicOr(p.status, SPECVLM_STATUS_TIMEOUT);
+  if (warp >= kSoftmaxWarp0 && !aborted && landed) {
+    if (inputs_stable) pdl_wait();  // `out` may still be in use by the preceding kernel
+#pragma unroll 1
+    for (int k = sw; k < rk; k += 4) {
+      const int row = split + k * ns;
+      if (row >= T) break;
+      // every lane reads all (max, sum) pairs of the row (broadcast loads) and four columns of each partial
+      float m[8], l[8];
       float4 x[8];
+      float mstar = -INFINITY;
 #pragma unroll
-      for (int s = 0; s < 8; ++s)
-        if (s < nsplit) x[s] = *(reinterpret_cast<const float4*>(cluster.map_shared_rank(so, s) + row * kD) + lane);
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int s = 0; s < 8; ++s) {
-        const float ws = __shfl_sync(0xffffffffu, w, s);
-        if (s < nsplit && ws > 0.f) {
-          acc.x += ws * x[s].x; acc.y += ws * x[s].y; acc.z += ws * x[s].z; acc.w += ws * x[s].w;
+      for (int s2 = 0; s2 < 8; ++s2) {
+        m[s2] = -INFINITY; l[s2] = 0.f; x[s2] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (s2 < ns) {
+          const float* src = (s2 == split ? stage + split * rk * kLandStride : landp + s2 * rk * kLandStride) + k * kLandStride;
+          const float2 ml = *reinterpret_cast<const float2*>(src + kD);
+          m[s2] = ml.x; l[s2] = ml.y;
+          x[s2] = *(reinterpret_cast<const float4*>(src) + lane);
+          mstar = fmaxf(mstar, ml.x);
         }
+      }
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float lsum = 0.f;
+#pragma unroll
+      for (int s2 = 0; s2 < 8; ++s2) {
+        const float w = (m[s2] == -INFINITY) ? 0.f : ex2(m[s2] - mstar);
+        lsum += w * l[s2];
+        acc.x += w * x[s2].x; acc.y += w * x[s2].y; acc.z += w * x[s2].z; acc.w += w * x[s2].w;
       }
       const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
       uint2 packed;
@@ -552,7 +740,10 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
       *reinterpret_cast<uint2*>(obase + row * p.o_st + lane * 4) = packed;
     }
   }
-  cluster.sync();  // nobody leaves while its shared memory may still be read
+#ifdef SPECVLM_TC_TRACE
+  if (warp == 2) TRACE(46);
+#endif
+  cluster.barrier_wait();
 }
 
 // ------------------------------------------------------------------ host side
@@ -598,12 +789,12 @@ int make_map(CUtensorMap* map, const void* base, int rows, int dim2, int dim3, i
 
 bool attn_tc_available() { return encode_fn() != nullptr; }
 
-int launch_attn_tc(const AttnParams& p, const specvlm_attn_desc& d, cudaStream_t stream) {
-  if (!attn_tc_available()) return fail(SPECVLM_ERR_UNSUPPORTED, "tensor-map encoder not available from the driver");
+template <class C>
+static int launch_cfg(const AttnParams& p, const specvlm_attn_desc& d, cudaStream_t stream) {
   CUtensorMap mq, mk, mv;
   int rc = make_map(&mq, p.q, d.T, d.H, d.B, d.q_stride_t, d.q_stride_h, d.q_stride_b, tc::kRows);
-  if (rc == SPECVLM_OK) rc = make_map(&mk, p.k, d.S_cap, d.H, d.B, d.k_stride_s, d.k_stride_h, d.k_stride_b, tc::kTile);
-  if (rc == SPECVLM_OK) rc = make_map(&mv, p.v, d.S_cap, d.H, d.B, d.v_stride_s, d.v_stride_h, d.v_stride_b, tc::kTile);
+  if (rc == SPECVLM_OK) rc = make_map(&mk, p.k, d.S_cap, d.H, d.B, d.k_stride_s, d.k_stride_h, d.k_stride_b, C::kTile);
+  if (rc == SPECVLM_OK) rc = make_map(&mv, p.v, d.S_cap, d.H, d.B, d.v_stride_s, d.v_stride_h, d.v_stride_b, C::kTile);
   if (rc != SPECVLM_OK) return rc;
 
   static bool attr_set[64] = {};
@@ -611,8 +802,8 @@ int launch_attn_tc(const AttnParams& p, const specvlm_attn_desc& d, cudaStream_t
   rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
   if (rc != SPECVLM_OK) return rc;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    rc = check_cuda(cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         tc::kSmemBytes),
+    rc = check_cuda(cudaFuncSetAttribute(tree_attn_tc_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         C::kSmemBytes),
                     "attn (tcgen05) smem attribute");
     if (rc != SPECVLM_OK) return rc;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
@@ -620,16 +811,32 @@ int launch_attn_tc(const AttnParams& p, const specvlm_attn_desc& d, cudaStream_t
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p.splits, d.H, d.B);
   cfg.blockDim = dim3(tc::kThreads);
-  cfg.dynamicSmemBytes = tc::kSmemBytes;
+  cfg.dynamicSmemBytes = C::kSmemBytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = p.splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // The kernel may be scheduled while the preceding kernel on the stream drains; it orders its own
+  // reads and writes with griddepcontrol.wait according to the descriptor flags.
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return check_cuda(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, p, mq, mk, mv), "tree_verify_attn (tcgen05) launch");
+  cfg.numAttrs = 2;
+  return check_cuda(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<C>, p, mq, mk, mv), "tree_verify_attn (tcgen05) launch");
+}
+
+int attn_tc_tile(const specvlm_attn_desc& d) {
+  return (d.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) ? tc::CfgThroughput::kTile : tc::CfgLatency::kTile;
+}
+
+int launch_attn_tc(const AttnParams& p, const specvlm_attn_desc& d, cudaStream_t stream) {
+  if (!attn_tc_available()) return fail(SPECVLM_ERR_UNSUPPORTED, "tensor-map encoder not available from the driver");
+  // Launches that the caller declares independent of their predecessor run in the half-SM
+  // configuration so that consecutive launches overlap; all others get the whole SM.
+  if (d.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) return launch_cfg<tc::CfgThroughput>(p, d, stream);
+  return launch_cfg<tc::CfgLatency>(p, d, stream);
 }
 
 }  // namespace specvlm

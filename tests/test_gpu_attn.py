@@ -12,12 +12,14 @@ from util import (ATTN_MAX_ABS, ATTN_MEAN_ABS, assert_attn_close, bits_to_torch,
 
 pytestmark = pytest.mark.gpu
 
-# Every test in this file runs twice: on the default (tcgen05) kernel and on the legacy
-# mma.sync kernels selected through the descriptor flag.
+# Every test in this file runs on each kernel variant, selected through the descriptor flags:
+# the whole-SM tcgen05 configuration (default), the half-SM tcgen05 configuration used for
+# launches declared independent of their predecessor, and the legacy mma.sync kernels.
 ATTN_FLAGS = 0
 
 
-@pytest.fixture(autouse=True, params=[0, sv.ATTN_FLAG_LEGACY_MMA], ids=["tcgen05", "legacy_mma"])
+@pytest.fixture(autouse=True, params=[0, sv.ATTN_FLAG_INPUTS_STABLE, sv.ATTN_FLAG_PREFIX_STABLE, sv.ATTN_FLAG_LEGACY_MMA],
+                ids=["tcgen05_full_sm", "tcgen05_half_sm", "tcgen05_prefix_prefetch", "legacy_mma"])
 def _attn_path(request):
     global ATTN_FLAGS
     ATTN_FLAGS = request.param
