@@ -276,9 +276,11 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
                  "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // The next launch on the stream may begin its own set-up now; it decides itself what it may read.
+  // Without a promise from the caller, nothing below may run before the preceding kernel has
+  // completed. Only then is the next launch allowed to start: a successor that was promised stable
+  // inputs must not overtake work that this kernel itself still had to wait for.
+  if (!prefix_stable) pdl_wait();
   pdl_launch_dependents();
-  if (!prefix_stable) pdl_wait();  // everything below reads memory the preceding kernel may have written
   const int prefix_raw = p.prefix_len[b];
   tc_fence_before();
   __syncthreads();
