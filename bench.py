@@ -413,13 +413,13 @@ def run_ours(args, cfg):
         achieved = kv_bytes_per_launch / attn_s_per_launch / 1e9
         ser_attn_s = ser_attn_ms * 1e-3 / (args.steps * L)
         ser_gbs = kv_bytes_per_launch / ser_attn_s / 1e9
-        traffic = None
-        prof = os.path.join(ROOT, "profiles", "attn_traffic.json")
+        traffic = None   # measured DRAM bytes per attention launch, from the ncu summary under profiles/
+        prof = os.path.join(ROOT, "profiles", f"attn_traffic_{cfg.name}.txt")
         if os.path.exists(prof):
-            try:
-                traffic = json.load(open(prof)).get(cfg.name)
-            except Exception:
-                traffic = None
+            for ln in open(prof):
+                parts = ln.split()
+                if len(parts) == 2 and parts[0] == cfg.name and parts[1].isdigit():
+                    traffic = int(parts[1])
         line = {
             "metric": METRIC, "value": world * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
