@@ -655,20 +655,23 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
   if (warp >= kSoftmaxWarp0 && !aborted0) {
     float* d0 = stage + ((row0 % ns) * rk + row0 / ns) * kLandStride + t4 * 2;
     float* d1 = stage + ((row1 % ns) * rk + row1 / ns) * kLandStride + t4 * 2;
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-      float ov[16];
-      if (have_o) {
-        tmem_ld32(to0 + c * 32, ov);
-        tmem_wait_ld();
-      } else {
+    float ov[4][16];
+    if (have_o) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) ov[j] = 0.f;
-      }
+      for (int c = 0; c < 4; ++c) tmem_ld32(to0 + c * 32, ov[c]);
+      tmem_wait_ld();
+    } else {
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int j = 0; j < 16; ++j) ov[c][j] = 0.f;
+    }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        *reinterpret_cast<float2*>(d0 + c * 32 + j * 8) = make_float2(ov[4 * j + 0], ov[4 * j + 1]);
-        *reinterpret_cast<float2*>(d1 + c * 32 + j * 8) = make_float2(ov[4 * j + 2], ov[4 * j + 3]);
+        *reinterpret_cast<float2*>(d0 + c * 32 + j * 8) = make_float2(ov[c][4 * j + 0], ov[c][4 * j + 1]);
+        *reinterpret_cast<float2*>(d1 + c * 32 + j * 8) = make_float2(ov[c][4 * j + 2], ov[c][4 * j + 3]);
       }
     }
     if (t4 == 0) {
@@ -708,38 +711,44 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
   if (aborted && threadIdx.x == 0 && p.status != nullptr) atomicOr(p.status, SPECVLM_STATUS_TIMEOUT);
   if (warp >= kSoftmaxWarp0 && !aborted && landed) {
     if (inputs_stable) pdl_wait();  // `out` may still be in use by the preceding kernel
+    // A warp pass covers four owned rows (k = sw + 4 rr + 16 pass); lane (rr, cc) combines 16 columns.
+    const int rr = lane >> 3, cc = lane & 7;
 #pragma unroll 1
-    for (int k = sw; k < rk; k += 4) {
+    for (int k = sw + 4 * rr; k < rk; k += 16) {
       const int row = split + k * ns;
-      if (row >= T) break;
-      // every lane reads all (max, sum) pairs of the row (broadcast loads) and four columns of each partial
-      float m[8], l[8];
-      float4 x[8];
-      float mstar = -INFINITY;
+      if (row < T) {
+        float mstar = -INFINITY;
+#pragma unroll 1
+        for (int s2 = 0; s2 < ns; ++s2) {
+          const float* src = (s2 == split ? stage + split * rk * kLandStride : landp + s2 * rk * kLandStride) + k * kLandStride;
+          mstar = fmaxf(mstar, src[kD]);
+        }
+        float4 acc[4];
 #pragma unroll
-      for (int s2 = 0; s2 < 8; ++s2) {
-        m[s2] = -INFINITY; l[s2] = 0.f; x[s2] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (s2 < ns) {
+        for (int q4 = 0; q4 < 4; ++q4) acc[q4] = make_float4(0.f, 0.f, 0.f, 0.f);
+        float lsum = 0.f;
+#pragma unroll 1
+        for (int s2 = 0; s2 < ns; ++s2) {
           const float* src = (s2 == split ? stage + split * rk * kLandStride : landp + s2 * rk * kLandStride) + k * kLandStride;
           const float2 ml = *reinterpret_cast<const float2*>(src + kD);
-          m[s2] = ml.x; l[s2] = ml.y;
-          x[s2] = *(reinterpret_cast<const float4*>(src) + lane);
-          mstar = fmaxf(mstar, ml.x);
-        }
-      }
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      float lsum = 0.f;
+          const float w = (ml.x == -INFINITY) ? 0.f : ex2(ml.x - mstar);
+          lsum += w * ml.y;
 #pragma unroll
-      for (int s2 = 0; s2 < 8; ++s2) {
-        const float w = (m[s2] == -INFINITY) ? 0.f : ex2(m[s2] - mstar);
-        lsum += w * l[s2];
-        acc.x += w * x[s2].x; acc.y += w * x[s2].y; acc.z += w * x[s2].z; acc.w += w * x[s2].w;
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const float4 x = *(reinterpret_cast<const float4*>(src + cc * 16) + q4);
+            acc[q4].x += w * x.x; acc[q4].y += w * x.y; acc[q4].z += w * x.z; acc[q4].w += w * x.w;
+          }
+        }
+        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+        uint4 lo, hi;
+        lo.x = pack_bf16(acc[0].x * inv, acc[0].y * inv); lo.y = pack_bf16(acc[0].z * inv, acc[0].w * inv);
+        lo.z = pack_bf16(acc[1].x * inv, acc[1].y * inv); lo.w = pack_bf16(acc[1].z * inv, acc[1].w * inv);
+        hi.x = pack_bf16(acc[2].x * inv, acc[2].y * inv); hi.y = pack_bf16(acc[2].z * inv, acc[2].w * inv);
+        hi.z = pack_bf16(acc[3].x * inv, acc[3].y * inv); hi.w = pack_bf16(acc[3].z * inv, acc[3].w * inv);
+        uint4* dst = reinterpret_cast<uint4*>(obase + row * p.o_st + cc * 16);
+        dst[0] = lo;
+        dst[1] = hi;
       }
-      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-      uint2 packed;
-      packed.x = pack_bf16(acc.x * inv, acc.y * inv);
-      packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-      *reinterpret_cast<uint2*>(obase + row * p.o_st + lane * 4) = packed;
     }
   }
 #ifdef SPECVLM_TC_TRACE
