@@ -105,6 +105,18 @@ typedef struct specvlm_kv_desc {
   int64_t stride_l, stride_b, stride_h, stride_s; /* same for K and V */
 } specvlm_kv_desc;
 
+/* Shapes and strides (in ELEMENTS) of the RoPE + append call for one layer. */
+typedef struct specvlm_rope_desc {
+  int32_t B, H, T, D, S_cap; /* D must be 128 */
+  float rope_base;           /* 0 = 10000 */
+  int64_t qi_stride_b, qi_stride_h, qi_stride_t; /* q_in   [B][H][T][D] */
+  int64_t kn_stride_b, kn_stride_h, kn_stride_t; /* k_new  [B][H][T][D] */
+  int64_t vn_stride_b, vn_stride_h, vn_stride_t; /* v_new  [B][H][T][D] */
+  int64_t qo_stride_b, qo_stride_h, qo_stride_t; /* q_out  [B][H][T][D] */
+  int64_t kc_stride_b, kc_stride_h, kc_stride_s; /* k_cache [B][H][S_cap][D] */
+  int64_t vc_stride_b, vc_stride_h, vc_stride_s; /* v_cache [B][H][S_cap][D] */
+} specvlm_rope_desc;
+
 SPECVLM_API int specvlm_version(void);
 SPECVLM_API const char* specvlm_last_error_string(void);
 
@@ -134,6 +146,23 @@ SPECVLM_API int specvlm_tree_build(const int32_t* tree_parent, const int32_t* pr
  * Returns SPECVLM_OK or SPECVLM_ERR_BAD_TREE. */
 SPECVLM_API int specvlm_tree_validate_host(const int32_t* tree_parent_host, const int32_t* draft_tokens_host,
                                int T);
+
+/*
+ * Positioned inputs for tree attention (Section 4.1; the LLaVA targets of Section 4.1 are
+ * LLaMA/Vicuna decoders with rotary position embedding). For every sequence b, head h and
+ * tree node t, with pos = prefix_len[b] + depth(t):
+ *     q_out[b][h][t]                       = RoPE(q_in[b][h][t], pos)
+ *     k_cache[b][h][prefix_len[b] + t]     = RoPE(k_new[b][h][t], pos)
+ *     v_cache[b][h][prefix_len[b] + t]     = v_new[b][h][t]
+ * RoPE rotates the pairs (d, d + 64) by the angle pos * base^(-2d/128). bf16 in and out,
+ * angles reduced in double, rotation in fp32. q_out may alias q_in. No other cache byte is
+ * written. pos_out (int32 [B][T], may be NULL) receives the position ids. A malformed tree or
+ * a prefix that does not fit sets status bits and skips that sequence.
+ */
+SPECVLM_API int specvlm_rope_append(const uint16_t* q_in, const uint16_t* k_new, const uint16_t* v_new,
+                        const int32_t* prefix_len, const int32_t* tree_parent, uint16_t* q_out,
+                        uint16_t* k_cache, uint16_t* v_cache, const specvlm_rope_desc* desc_host,
+                        int32_t* pos_out, int32_t* status, void* stream);
 
 /*
  * Tree-verification attention for ONE layer (Sections 3.1, 3.2, 4.1).

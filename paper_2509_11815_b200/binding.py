@@ -29,6 +29,7 @@ EXPORTS = (
     "specvlm_tree_validate_host",
     "specvlm_tree_verify_attn",
     "specvlm_tree_verify_attn_static",
+    "specvlm_rope_append",
     "specvlm_argmax",
     "specvlm_accept",
     "specvlm_kv_compact",
@@ -59,6 +60,14 @@ class KvDesc(ctypes.Structure):
         ("stride_l", ctypes.c_int64), ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64),
         ("stride_s", ctypes.c_int64),
     ]
+
+
+class RopeDesc(ctypes.Structure):
+    _fields_ = ([("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("D", ctypes.c_int32),
+                 ("S_cap", ctypes.c_int32), ("rope_base", ctypes.c_float)] +
+                [(f"{n}_stride_{a}", ctypes.c_int64) for n, axes in (("qi", "bht"), ("kn", "bht"), ("vn", "bht"),
+                                                                      ("qo", "bht"), ("kc", "bhs"), ("vc", "bhs"))
+                 for a in axes])
 
 
 _lib = None
@@ -92,6 +101,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.specvlm_tree_verify_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(AttnDesc), vp, vp, vp]
     lib.specvlm_tree_verify_attn_static.restype = i32
     lib.specvlm_tree_verify_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(AttnDesc), vp, vp]
+    lib.specvlm_rope_append.restype = i32
+    lib.specvlm_rope_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(RopeDesc), vp, vp, vp]
     lib.specvlm_argmax.restype = i32
     lib.specvlm_argmax.argtypes = [vp, i32, i32, i32, i64, vp, vp]
     lib.specvlm_accept.restype = i32
@@ -242,6 +253,33 @@ def specvlm_tree_verify_attn_static(q: torch.Tensor, k_cache: torch.Tensor, v_ca
     _check(load_library().specvlm_tree_verify_attn_static(
         _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(prefix_len), _ptr(tree_parent), _ptr(tree_mask_bits),
         _ptr(out), ctypes.byref(desc), _ptr(status), _stream()))
+
+
+def specvlm_rope_append(q_in: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, prefix_len: torch.Tensor,
+                        tree_parent: torch.Tensor, q_out: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                        pos_out: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+                        rope_base: float = 0.0) -> None:
+    """RoPE of q and the tree's new K rows at prefix_len + depth, and append of the tree's K/V rows
+    to one layer's cache. q_in/k_new/v_new/q_out: [B][H][T][D]; k_cache/v_cache: [B][H][S_cap][D]."""
+    for name, t in (("q_in", q_in), ("k_new", k_new), ("v_new", v_new), ("q_out", q_out), ("k_cache", k_cache),
+                    ("v_cache", v_cache)):
+        _need(t, torch.bfloat16, name)
+        if t.dim() != 4 or t.stride(3) != 1:
+            raise SpecvlmError(f"{name} must be 4-D with a contiguous last dimension")
+    _need(prefix_len, torch.int32, "prefix_len")
+    _need(tree_parent, torch.int32, "tree_parent")
+    B, H, T, D = q_in.shape
+    d = RopeDesc()
+    d.B, d.H, d.T, d.D, d.S_cap, d.rope_base = B, H, T, D, k_cache.shape[2], rope_base
+    for n, t in (("qi", q_in), ("kn", k_new), ("vn", v_new), ("qo", q_out)):
+        for a, i in (("b", 0), ("h", 1), ("t", 2)):
+            setattr(d, f"{n}_stride_{a}", t.stride(i))
+    for n, t in (("kc", k_cache), ("vc", v_cache)):
+        for a, i in (("b", 0), ("h", 1), ("s", 2)):
+            setattr(d, f"{n}_stride_{a}", t.stride(i))
+    _check(load_library().specvlm_rope_append(_ptr(q_in), _ptr(k_new), _ptr(v_new), _ptr(prefix_len),
+                                              _ptr(tree_parent), _ptr(q_out), _ptr(k_cache), _ptr(v_cache),
+                                              ctypes.byref(d), _ptr(pos_out), _ptr(status), _stream()))
 
 
 def specvlm_argmax(target_logits: torch.Tensor, argmax_tokens: torch.Tensor) -> None:
