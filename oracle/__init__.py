@@ -27,3 +27,4 @@ from .accept import (  # noqa: F401
     accept_bruteforce,
     kv_compact,
 )
+from .sample import accept_sample, decision_margins, softmax_f64  # noqa: F401
