@@ -246,6 +246,26 @@ SPECVLM_API int specvlm_accept(const int32_t* draft_tokens, const int32_t* tree_
                    int32_t* next_token, int32_t* status, void* stream);
 
 /*
+ * Temperature > 0 acceptance by speculative sampling on the tree (Section 3.1: speculative
+ * sampling discards incorrect tokens; Section 4.1: stochastic decoding, target distribution
+ * preserved). Children are fixed candidates tried in index order: at the current node with
+ * p = softmax(target_logits / temperature), child c with token x is kept iff
+ * uniforms_accept[b][c] < p(x) / (1 - mass already rejected at this node); a rejected token is
+ * removed from p. If a child is kept the walk descends to it; otherwise next_token is drawn
+ * from what is left of p by inverse CDF with uniforms_sample[b][node] (also at a kept leaf).
+ *   target_logits    fp32 [B][T][V] contiguous
+ *   uniforms_accept  fp32 [B][T] in [0, 1): entry c is used for the keep test of node c
+ *   uniforms_sample  fp32 [B][T] in [0, 1): entry u is used if the walk stops at node u
+ *   outputs as in specvlm_accept. fp32 arithmetic; a decision whose random number lies within
+ *   rounding distance of its threshold may differ from an exact evaluation.
+ */
+SPECVLM_API int specvlm_accept_sample(const int32_t* draft_tokens, const int32_t* tree_parent,
+                          const float* target_logits, const float* uniforms_accept,
+                          const float* uniforms_sample, float temperature, int B, int T, int V,
+                          int32_t* accepted_idx, int acc_stride, int32_t* accept_len,
+                          int32_t* next_token, int32_t* status, void* stream);
+
+/*
  * KV compaction after acceptance (the KV cache is the resource the paper's cost model
  * is about, Sections 1 and 3.2). For every layer, for K and V, for every (b, h) and
  * j = 1..accept_len[b]: the 256-byte row in slot prefix_len[b] + accepted_idx[b][j] moves

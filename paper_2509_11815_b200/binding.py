@@ -32,6 +32,7 @@ EXPORTS = (
     "specvlm_rope_append",
     "specvlm_argmax",
     "specvlm_accept",
+    "specvlm_accept_sample",
     "specvlm_kv_compact",
     "specvlm_accept_compact",
 )
@@ -107,6 +108,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.specvlm_argmax.argtypes = [vp, i32, i32, i32, i64, vp, vp]
     lib.specvlm_accept.restype = i32
     lib.specvlm_accept.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, i32, vp, vp, vp, vp]
+    lib.specvlm_accept_sample.restype = i32
+    lib.specvlm_accept_sample.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, i32, i32, i32, vp, i32, vp, vp, vp, vp]
     lib.specvlm_kv_compact.restype = i32
     lib.specvlm_kv_compact.argtypes = [vp, vp, ctypes.POINTER(KvDesc), vp, vp, i32, vp, vp, vp, vp]
     lib.specvlm_accept_compact.restype = i32
@@ -309,6 +312,26 @@ def specvlm_accept(draft_tokens: torch.Tensor, tree_parent: torch.Tensor, target
     _check(load_library().specvlm_accept(_ptr(draft_tokens), _ptr(tree_parent), _ptr(target_logits),
                                          _ptr(argmax_tokens), B, T, V, _ptr(accepted_idx), accepted_idx.shape[1],
                                          _ptr(accept_len), _ptr(next_token), _ptr(status), _stream()))
+
+
+def specvlm_accept_sample(draft_tokens: torch.Tensor, tree_parent: torch.Tensor, target_logits: torch.Tensor,
+                          uniforms_accept: torch.Tensor, uniforms_sample: torch.Tensor, temperature: float,
+                          accepted_idx: torch.Tensor, accept_len: torch.Tensor, next_token: torch.Tensor,
+                          status: Optional[torch.Tensor] = None) -> None:
+    """Temperature > 0 tree acceptance by speculative sampling; see include/specvlm.h."""
+    for name, t in (("draft_tokens", draft_tokens), ("tree_parent", tree_parent), ("accepted_idx", accepted_idx),
+                    ("accept_len", accept_len), ("next_token", next_token)):
+        _need(t, torch.int32, name)
+    for name, t in (("target_logits", target_logits), ("uniforms_accept", uniforms_accept),
+                    ("uniforms_sample", uniforms_sample)):
+        _need(t, torch.float32, name)
+        if not t.is_contiguous():
+            raise SpecvlmError(f"{name} must be contiguous")
+    B, T = draft_tokens.shape
+    _check(load_library().specvlm_accept_sample(
+        _ptr(draft_tokens), _ptr(tree_parent), _ptr(target_logits), _ptr(uniforms_accept), _ptr(uniforms_sample),
+        float(temperature), B, T, target_logits.shape[-1], _ptr(accepted_idx), accepted_idx.shape[1],
+        _ptr(accept_len), _ptr(next_token), _ptr(status), _stream()))
 
 
 def make_kv_desc(cache: torch.Tensor) -> KvDesc:
