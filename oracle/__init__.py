@@ -28,3 +28,4 @@ from .accept import (  # noqa: F401
     kv_compact,
 )
 from .sample import accept_sample, decision_margins, softmax_f64  # noqa: F401
+from .draft_tree import rerank_tree, topk_logprob  # noqa: F401
