@@ -148,6 +148,36 @@ SPECVLM_API int specvlm_tree_validate_host(const int32_t* tree_parent_host, cons
                                int T);
 
 /*
+ * Draft-tree construction, step 1 (Section 4.1: top-k 10 expansion): for each of `rows` logits
+ * rows (row r starts at logits + r * row_stride, fp32, V entries) the k <= 16 most probable
+ * tokens in order (ties: lower token id first) and their log-probabilities
+ * log softmax(logits)[token].
+ *   tokens int32 [rows][k] out, logprob fp32 [rows][k] out
+ */
+SPECVLM_API int specvlm_topk_logprob(const float* logits, int rows, int V, int64_t row_stride, int k,
+                         int32_t* tokens, float* logprob, void* stream);
+
+/*
+ * Draft-tree construction, step 2 (Section 4.1: 60 tokens in total): rerank of all candidates
+ * by cumulative score. Candidate 0 is the root (cand_parent = -1), cand_parent[c] < c.
+ * The root and the T-1 best-scoring other candidates are kept (ties: lower candidate index
+ * first) and relabelled in (depth, score descending, candidate index) order, so that
+ * parent < child.
+ *   cand_parent int32 [B][C], cand_score fp32 [B][C] (cumulative log-probability, compared
+ *   exactly), cand_token int32 [B][C]; T <= C <= 1024
+ *   tree_parent int32 [B][T] out, draft_tokens int32 [B][T] out
+ *   kept_candidates int32 [B][T] out (may be NULL): candidate id of every tree node
+ *   mask_bits uint64 [B][T], depth int32 [B][T], pos int32 [B][T] out (each may be NULL;
+ *   pos = prefix_len[b] + depth needs prefix_len)
+ * Scores must not increase from parent to child (log-probabilities are <= 0); otherwise a kept
+ * node's parent may be missing and SPECVLM_STATUS_BAD_TREE is set.
+ */
+SPECVLM_API int specvlm_tree_rerank(const int32_t* cand_parent, const float* cand_score, const int32_t* cand_token,
+                        const int32_t* prefix_len, int B, int C, int T, int32_t* tree_parent,
+                        int32_t* draft_tokens, int32_t* kept_candidates, uint64_t* mask_bits,
+                        int32_t* depth, int32_t* pos, int32_t* status, void* stream);
+
+/*
  * Positioned inputs for tree attention (Section 4.1; the LLaVA targets of Section 4.1 are
  * LLaMA/Vicuna decoders with rotary position embedding). For every sequence b, head h and
  * tree node t, with pos = prefix_len[b] + depth(t):

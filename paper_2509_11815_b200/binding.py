@@ -29,6 +29,8 @@ EXPORTS = (
     "specvlm_tree_validate_host",
     "specvlm_tree_verify_attn",
     "specvlm_tree_verify_attn_static",
+    "specvlm_topk_logprob",
+    "specvlm_tree_rerank",
     "specvlm_rope_append",
     "specvlm_argmax",
     "specvlm_accept",
@@ -102,6 +104,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.specvlm_tree_verify_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(AttnDesc), vp, vp, vp]
     lib.specvlm_tree_verify_attn_static.restype = i32
     lib.specvlm_tree_verify_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(AttnDesc), vp, vp]
+    lib.specvlm_topk_logprob.restype = i32
+    lib.specvlm_topk_logprob.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp]
+    lib.specvlm_tree_rerank.restype = i32
+    lib.specvlm_tree_rerank.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.specvlm_rope_append.restype = i32
     lib.specvlm_rope_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(RopeDesc), vp, vp, vp]
     lib.specvlm_argmax.restype = i32
@@ -256,6 +262,32 @@ def specvlm_tree_verify_attn_static(q: torch.Tensor, k_cache: torch.Tensor, v_ca
     _check(load_library().specvlm_tree_verify_attn_static(
         _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(prefix_len), _ptr(tree_parent), _ptr(tree_mask_bits),
         _ptr(out), ctypes.byref(desc), _ptr(status), _stream()))
+
+
+def specvlm_topk_logprob(logits: torch.Tensor, k: int, tokens: torch.Tensor, logprob: torch.Tensor) -> None:
+    """logits fp32 [rows][V] (row-strided), tokens int32 [rows][k], logprob fp32 [rows][k]."""
+    _need(logits, torch.float32, "logits")
+    _need(tokens, torch.int32, "tokens")
+    _need(logprob, torch.float32, "logprob")
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise SpecvlmError("logits must be [rows][V] with a contiguous last dimension")
+    _check(load_library().specvlm_topk_logprob(_ptr(logits), logits.shape[0], logits.shape[1], logits.stride(0), k,
+                                               _ptr(tokens), _ptr(logprob), _stream()))
+
+
+def specvlm_tree_rerank(cand_parent: torch.Tensor, cand_score: torch.Tensor, cand_token: torch.Tensor, T: int,
+                        tree_parent: torch.Tensor, draft_tokens: torch.Tensor,
+                        kept_candidates: Optional[torch.Tensor] = None, mask_bits: Optional[torch.Tensor] = None,
+                        depth: Optional[torch.Tensor] = None, pos: Optional[torch.Tensor] = None,
+                        prefix_len: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None) -> None:
+    """Rerank [B][C] candidates into [B][T] trees; see include/specvlm.h."""
+    _need(cand_parent, torch.int32, "cand_parent")
+    _need(cand_score, torch.float32, "cand_score")
+    _need(cand_token, torch.int32, "cand_token")
+    B, C = cand_parent.shape
+    _check(load_library().specvlm_tree_rerank(_ptr(cand_parent), _ptr(cand_score), _ptr(cand_token), _ptr(prefix_len),
+                                              B, C, T, _ptr(tree_parent), _ptr(draft_tokens), _ptr(kept_candidates),
+                                              _ptr(mask_bits), _ptr(depth), _ptr(pos), _ptr(status), _stream()))
 
 
 def specvlm_rope_append(q_in: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, prefix_len: torch.Tensor,
