@@ -29,3 +29,4 @@ from .accept import (  # noqa: F401
 )
 from .sample import accept_sample, decision_margins, softmax_f64  # noqa: F401
 from .draft_tree import rerank_tree, topk_logprob  # noqa: F401
+from .compress import visual_pool, visual_prune  # noqa: F401
