@@ -148,6 +148,19 @@ SPECVLM_API int specvlm_tree_validate_host(const int32_t* tree_parent_host, cons
                                int T);
 
 /*
+ * Parameter-free visual token compression (Section 3.4: pooling and random pruning of the
+ * elastic compressor). x: bf16 [B][N][C] visual tokens, C a multiple of 8, contiguous.
+ * specvlm_visual_pool: y[b][m] = mean of x[b][m*ratio .. min((m+1)*ratio, N)), fp32
+ *   accumulation; y: bf16 [B][ceil(N/ratio)][C].
+ * specvlm_visual_prune: y[b][m] = x[b][keep_idx[b][m]] bit for bit (the random choice of the kept
+ *   tokens is the caller's input); y: bf16 [B][M][C]; an index outside [0, N) yields a zero row
+ *   and sets SPECVLM_STATUS_BAD_ACCEPT.
+ */
+SPECVLM_API int specvlm_visual_pool(const uint16_t* x, int B, int N, int C, int ratio, uint16_t* y, void* stream);
+SPECVLM_API int specvlm_visual_prune(const uint16_t* x, const int32_t* keep_idx, int B, int N, int C, int M,
+                         uint16_t* y, int32_t* status, void* stream);
+
+/*
  * Draft-tree construction, step 1 (Section 4.1: top-k 10 expansion): for each of `rows` logits
  * rows (row r starts at logits + r * row_stride, fp32, V entries) the k <= 16 most probable
  * tokens in order (ties: lower token id first) and their log-probabilities

@@ -29,6 +29,8 @@ EXPORTS = (
     "specvlm_tree_validate_host",
     "specvlm_tree_verify_attn",
     "specvlm_tree_verify_attn_static",
+    "specvlm_visual_pool",
+    "specvlm_visual_prune",
     "specvlm_topk_logprob",
     "specvlm_tree_rerank",
     "specvlm_rope_append",
@@ -104,6 +106,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.specvlm_tree_verify_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(AttnDesc), vp, vp, vp]
     lib.specvlm_tree_verify_attn_static.restype = i32
     lib.specvlm_tree_verify_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(AttnDesc), vp, vp]
+    lib.specvlm_visual_pool.restype = i32
+    lib.specvlm_visual_pool.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+    lib.specvlm_visual_prune.restype = i32
+    lib.specvlm_visual_prune.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp]
     lib.specvlm_topk_logprob.restype = i32
     lib.specvlm_topk_logprob.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp]
     lib.specvlm_tree_rerank.restype = i32
@@ -262,6 +268,31 @@ def specvlm_tree_verify_attn_static(q: torch.Tensor, k_cache: torch.Tensor, v_ca
     _check(load_library().specvlm_tree_verify_attn_static(
         _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(prefix_len), _ptr(tree_parent), _ptr(tree_mask_bits),
         _ptr(out), ctypes.byref(desc), _ptr(status), _stream()))
+
+
+def specvlm_visual_pool(x: torch.Tensor, ratio: int, y: torch.Tensor) -> None:
+    """x bf16 [B][N][C] contiguous -> y bf16 [B][ceil(N/ratio)][C]: window means over the token axis."""
+    _need(x, torch.bfloat16, "x")
+    _need(y, torch.bfloat16, "y")
+    if not (x.is_contiguous() and y.is_contiguous()):
+        raise SpecvlmError("x and y must be contiguous")
+    B, N, C = x.shape
+    if tuple(y.shape) != (B, (N + ratio - 1) // max(ratio, 1), C):
+        raise SpecvlmError("y must be [B][ceil(N/ratio)][C]")
+    _check(load_library().specvlm_visual_pool(_ptr(x), B, N, C, ratio, _ptr(y), _stream()))
+
+
+def specvlm_visual_prune(x: torch.Tensor, keep_idx: torch.Tensor, y: torch.Tensor,
+                         status: Optional[torch.Tensor] = None) -> None:
+    """x bf16 [B][N][C], keep_idx int32 [B][M] -> y bf16 [B][M][C]: the kept token rows."""
+    _need(x, torch.bfloat16, "x")
+    _need(y, torch.bfloat16, "y")
+    _need(keep_idx, torch.int32, "keep_idx")
+    if not (x.is_contiguous() and y.is_contiguous() and keep_idx.is_contiguous()):
+        raise SpecvlmError("x, y and keep_idx must be contiguous")
+    B, N, C = x.shape
+    M = keep_idx.shape[1]
+    _check(load_library().specvlm_visual_prune(_ptr(x), _ptr(keep_idx), B, N, C, M, _ptr(y), _ptr(status), _stream()))
 
 
 def specvlm_topk_logprob(logits: torch.Tensor, k: int, tokens: torch.Tensor, logprob: torch.Tensor) -> None:
