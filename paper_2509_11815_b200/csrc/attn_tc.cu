@@ -838,15 +838,15 @@ static int launch_cfg(const AttnParams& p, const specvlm_attn_desc& d, cudaStrea
   return check_cuda(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<C>, p, mq, mk, mv), "tree_verify_attn (tcgen05) launch");
 }
 
-int attn_tc_tile(const specvlm_attn_desc& d) {
-  return (d.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) ? tc::CfgThroughput::kTile : tc::CfgLatency::kTile;
-}
+int attn_tc_tile(const specvlm_attn_desc&) { return tc::CfgThroughput::kTile; }
 
 int launch_attn_tc(const AttnParams& p, const specvlm_attn_desc& d, cudaStream_t stream) {
   if (!attn_tc_available()) return fail(SPECVLM_ERR_UNSUPPORTED, "tensor-map encoder not available from the driver");
   // Launches that the caller declares independent of their predecessor run in the half-SM
-  // configuration so that consecutive launches overlap; all others get the whole SM.
-  if (d.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) return launch_cfg<tc::CfgThroughput>(p, d, stream);
+  // configuration so that consecutive launches overlap; so do launches with more CTAs than SMs,
+  // which would otherwise need a second wave. All others get the whole SM.
+  const int64_t ctas = static_cast<int64_t>(d.B) * d.H * p.splits;
+  if ((d.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) || ctas > sm_count()) return launch_cfg<tc::CfgThroughput>(p, d, stream);
   return launch_cfg<tc::CfgLatency>(p, d, stream);
 }
 
