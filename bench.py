@@ -272,9 +272,14 @@ def run_ours(args, cfg):
     #   pipelined : layers 1..L-1 are declared independent of the launch before them
     #               (SPECVLM_ATTN_FLAG_INPUTS_STABLE: their q / caches / out are not touched by it),
     #               so consecutive launches overlap through programmatic dependent launch.
-    #               Layer 0 stays serialized because the compaction kernel before it writes the caches.
+    #               Layer 0 waits for the compaction kernel before it (which writes tree slots of every
+    #               cache) but may prefetch its prefix tiles early (PREFIX_STABLE).
     desc_ser = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0])
     desc_pipe = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0], flags=sv.ATTN_FLAG_INPUTS_STABLE)
+    # layer 0 of a pipelined step: the compaction kernel before it only writes tree slots, so the
+    # prefix may be prefetched early; half-SM configuration so that layer 1 can overlap it
+    desc_pipe0 = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0],
+                                   flags=sv.ATTN_FLAG_PREFIX_STABLE | sv.ATTN_FLAG_HALF_SM)
     ws = sv.alloc_attn_workspace(desc_ser, dev)
     launches_per_step = L + 2
 
@@ -283,7 +288,7 @@ def run_ours(args, cfg):
         for l in range(L):
             sv.specvlm_tree_verify_attn(q[l], k_cache[l], v_cache[l], prefix_len, par, mask, out[l],
                                         workspace=ws, status=status,
-                                        desc=desc_pipe if (pipelined and l > 0) else desc_ser)
+                                        desc=(desc_pipe if l > 0 else desc_pipe0) if pipelined else desc_ser)
 
     def tail(i):
         par, drf, lg, mask = sets[i % N_INPUT_SETS]

@@ -78,6 +78,9 @@ extern "C" {
  *   attention calls on independent inputs, as in a benchmark). */
 #define SPECVLM_ATTN_FLAG_PREFIX_STABLE 2
 #define SPECVLM_ATTN_FLAG_INPUTS_STABLE 4
+/* Run in the configuration that occupies half an SM per thread block (chosen automatically for
+ * INPUTS_STABLE launches): use it for a launch that is followed by launches meant to overlap it. */
+#define SPECVLM_ATTN_FLAG_HALF_SM 8
 
 #define SPECVLM_MAX_TREE 64
 #define SPECVLM_HEAD_DIM 128

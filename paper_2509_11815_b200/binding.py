@@ -164,6 +164,7 @@ def specvlm_version() -> int:
 ATTN_FLAG_LEGACY_MMA = 1
 ATTN_FLAG_PREFIX_STABLE = 2
 ATTN_FLAG_INPUTS_STABLE = 4
+ATTN_FLAG_HALF_SM = 8
 
 
 def make_attn_desc(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,

@@ -426,7 +426,7 @@ int resolve_num_splits(const specvlm_attn_desc& d) {
       const int64_t target = 2 * static_cast<int64_t>(sm_count());
       splits = static_cast<int>((target + bh - 1) / bh);
       if (splits > kMaxClusterSplits && splits <= 2 * kMaxClusterSplits) splits = kMaxClusterSplits;
-    } else if (d.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) {
+    } else if (d.flags & (SPECVLM_ATTN_FLAG_INPUTS_STABLE | SPECVLM_ATTN_FLAG_HALF_SM)) {
       // launches overlap one another: few CTAs per launch, little or no split exchange
       splits = static_cast<int>((32 + bh - 1) / bh);
       if (splits > kMaxClusterSplits) splits = kMaxClusterSplits;

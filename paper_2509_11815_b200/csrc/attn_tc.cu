@@ -846,7 +846,8 @@ int launch_attn_tc(const AttnParams& p, const specvlm_attn_desc& d, cudaStream_t
   // configuration so that consecutive launches overlap; so do launches with more CTAs than SMs,
   // which would otherwise need a second wave. All others get the whole SM.
   const int64_t ctas = static_cast<int64_t>(d.B) * d.H * p.splits;
-  if ((d.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) || ctas > sm_count()) return launch_cfg<tc::CfgThroughput>(p, d, stream);
+  if ((d.flags & (SPECVLM_ATTN_FLAG_INPUTS_STABLE | SPECVLM_ATTN_FLAG_HALF_SM)) || ctas > sm_count())
+    return launch_cfg<tc::CfgThroughput>(p, d, stream);
   return launch_cfg<tc::CfgLatency>(p, d, stream);
 }
 

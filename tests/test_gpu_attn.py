@@ -18,8 +18,9 @@ pytestmark = pytest.mark.gpu
 ATTN_FLAGS = 0
 
 
-@pytest.fixture(autouse=True, params=[0, sv.ATTN_FLAG_INPUTS_STABLE, sv.ATTN_FLAG_PREFIX_STABLE, sv.ATTN_FLAG_LEGACY_MMA],
-                ids=["tcgen05_full_sm", "tcgen05_half_sm", "tcgen05_prefix_prefetch", "legacy_mma"])
+@pytest.fixture(autouse=True, params=[0, sv.ATTN_FLAG_INPUTS_STABLE, sv.ATTN_FLAG_PREFIX_STABLE, sv.ATTN_FLAG_PREFIX_STABLE | sv.ATTN_FLAG_HALF_SM,
+                        sv.ATTN_FLAG_LEGACY_MMA],
+                ids=["tcgen05_full_sm", "tcgen05_half_sm", "tcgen05_prefix_prefetch", "tcgen05_half_sm_prefix_prefetch", "legacy_mma"])
 def _attn_path(request):
     global ATTN_FLAGS
     ATTN_FLAGS = request.param

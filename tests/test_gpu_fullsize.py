@@ -1,7 +1,8 @@
 """GPU parity at the full workload sizes, in the launch configuration the benchmark times.
 
 All L layers are launched back to back on one stream exactly as bench.py does (layer 0
-serialized, layers 1..L-1 declared independent of the preceding launch so that they overlap),
+waiting for its predecessor with prefix prefetch, layers 1..L-1 declared independent of the
+preceding launch so that they overlap),
 followed by argmax and the fused accept + compaction launch. Attention is compared with the
 oracle on sampled (layer, sequence, head) outputs; argmax, acceptance and prefix lengths are
 compared in full (bit-exact); compaction is compared with the oracle on sampled (layer,
@@ -66,8 +67,10 @@ def run_verify_step(cfg_name, sampled_layers, heads_per_layer, seed_offset=0):
                               torch_to_bits(v_cache[l, b, h, :n])))
     k_before, v_before = k_cache.clone(), v_cache.clone()
 
-    desc_ser = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0])
+    desc_ser = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0])   # sizes the workspace
     desc_pipe = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0], flags=sv.ATTN_FLAG_INPUTS_STABLE)
+    desc_pipe0 = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0],
+                                   flags=sv.ATTN_FLAG_PREFIX_STABLE | sv.ATTN_FLAG_HALF_SM)
     ws = sv.alloc_attn_workspace(desc_ser, dev)
     tok = torch.zeros((B, T), **i32)
     acc_idx = torch.zeros((B, 8), **i32)
@@ -75,7 +78,7 @@ def run_verify_step(cfg_name, sampled_layers, heads_per_layer, seed_offset=0):
     torch.cuda.synchronize()
     for l in range(L):
         sv.specvlm_tree_verify_attn(q[l], k_cache[l], v_cache[l], prefix_len, par, mask, out[l], workspace=ws,
-                                    status=status, desc=desc_pipe if l > 0 else desc_ser)
+                                    status=status, desc=desc_pipe if l > 0 else desc_pipe0)
     sv.specvlm_argmax(lg, tok)
     sv.specvlm_accept_compact(drf, par, tok, k_cache, v_cache, prefix_len, acc_idx, acc_len, nxt, new_len, status)
     torch.cuda.synchronize()
