@@ -1,17 +1,19 @@
 // Vocabulary-wide argmax of the target logits at every tree node (the greedy target
 // token used by temperature-0 verification; part of the sampling cost of Eq. 1).
 //
-// One thread block per logits row. Every thread keeps the (value, lowest index) of the
-// maximum among the float4 groups it streams (128-bit coalesced loads), then the pairs
-// are reduced with "greater value, else lower index", which reproduces a sequential scan
-// with strict '>' bit for bit. HBM-bound: V * 4 bytes per row, read once.
+// One cluster of four thread blocks per logits row. Every thread keeps the (value, lowest
+// index) of the maximum among the float4 groups it streams (128-bit coalesced loads), then
+// the pairs are reduced with "greater value, else lower index", which reproduces a
+// sequential scan with strict '>' bit for bit. HBM-bound: V * 4 bytes per row, read once.
 #include "common.cuh"
 
+#include <cooperative_groups.h>
 #include <limits.h>
 
 namespace specvlm {
 
-constexpr int kArgmaxThreads = 512;
+constexpr int kArgmaxThreads = 256;
+constexpr int kArgmaxSplit = 4;  // CTAs per row = cluster size
 
 struct Best {
   float v;
@@ -30,55 +32,64 @@ __device__ __forceinline__ void take(Best& best, float v, int i) {
   }
 }
 
+// One cluster of kArgmaxSplit CTAs per logits row; each CTA scans a contiguous quarter of the
+// row's float4 groups, the partial (value, index) pairs meet in the first CTA's shared memory
+// through distributed shared memory.
 __global__ void __launch_bounds__(kArgmaxThreads)
 argmax_rows_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
                    int32_t* __restrict__ out) {
-  const int row = blockIdx.x;
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int row = blockIdx.y;
+  const int part = blockIdx.x;  // == rank in the cluster
   const float* x = logits + static_cast<int64_t>(row) * row_stride;
   const float4* x4 = reinterpret_cast<const float4*>(x);
   const int n4 = V >> 2;
+  const int per = (n4 + kArgmaxSplit - 1) / kArgmaxSplit;
+  const int g0 = part * per, g1 = min(g0 + per, n4);
 
+  cluster.barrier_arrive();  // matched by the wait below: every CTA of the cluster has started by then
   Best best{-INFINITY, INT_MAX};
   // -inf never passes '>' against the initial -inf; INT_MAX then loses every index tie,
   // and an all -inf row ends as index 0 below.
-  int g = threadIdx.x;
-  // Four independent 16-byte loads in flight per thread per trip.
-  for (; g + 3 * kArgmaxThreads < n4; g += 4 * kArgmaxThreads) {
-    float4 a = __ldcs(x4 + g);
-    float4 b = __ldcs(x4 + g + kArgmaxThreads);
-    float4 c = __ldcs(x4 + g + 2 * kArgmaxThreads);
-    float4 d = __ldcs(x4 + g + 3 * kArgmaxThreads);
-    int i = g * 4;
-    take(best, a.x, i); take(best, a.y, i + 1); take(best, a.z, i + 2); take(best, a.w, i + 3);
-    i = (g + kArgmaxThreads) * 4;
-    take(best, b.x, i); take(best, b.y, i + 1); take(best, b.z, i + 2); take(best, b.w, i + 3);
-    i = (g + 2 * kArgmaxThreads) * 4;
-    take(best, c.x, i); take(best, c.y, i + 1); take(best, c.z, i + 2); take(best, c.w, i + 3);
-    i = (g + 3 * kArgmaxThreads) * 4;
-    take(best, d.x, i); take(best, d.y, i + 1); take(best, d.z, i + 2); take(best, d.w, i + 3);
+  int g = g0 + threadIdx.x;
+  // Eight independent 16-byte loads in flight per thread per trip (a 32000-entry row is one trip).
+  for (; g < g1; g += 8 * kArgmaxThreads) {
+    float4 a[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int gu = g + u * kArgmaxThreads;
+      a[u] = (gu < g1) ? __ldcs(x4 + gu) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = (g + u * kArgmaxThreads) * 4;
+      take(best, a[u].x, i); take(best, a[u].y, i + 1); take(best, a[u].z, i + 2); take(best, a[u].w, i + 3);
+    }
   }
-  for (; g < n4; g += kArgmaxThreads) {
-    float4 a = __ldcs(x4 + g);
-    int i = g * 4;
-    take(best, a.x, i); take(best, a.y, i + 1); take(best, a.z, i + 2); take(best, a.w, i + 3);
-  }
-  for (int i = (n4 << 2) + threadIdx.x; i < V; i += kArgmaxThreads) take(best, x[i], i);
+  if (part == kArgmaxSplit - 1)  // the row's scalar tail belongs to the last part
+    for (int i = (n4 << 2) + threadIdx.x; i < V; i += kArgmaxThreads) take(best, x[i], i);
 
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
     Best o{__shfl_xor_sync(0xffffffffu, best.v, off), __shfl_xor_sync(0xffffffffu, best.i, off)};
     best = better(best, o);
   }
-  __shared__ float sv[kArgmaxThreads / 32];
-  __shared__ int si[kArgmaxThreads / 32];
+  constexpr int kWarps = kArgmaxThreads / 32;
+  __shared__ float sv[kArgmaxSplit * kWarps];
+  __shared__ int si[kArgmaxSplit * kWarps];
+  cluster.barrier_wait();
   if ((threadIdx.x & 31) == 0) {
-    sv[threadIdx.x >> 5] = best.v;
-    si[threadIdx.x >> 5] = best.i;
+    // every CTA deposits its warps' results in the first CTA's arrays
+    float* dv = cluster.map_shared_rank(sv, 0);
+    int* di = cluster.map_shared_rank(si, 0);
+    dv[part * kWarps + (threadIdx.x >> 5)] = best.v;
+    di[part * kWarps + (threadIdx.x >> 5)] = best.i;
   }
-  __syncthreads();
-  if (threadIdx.x < 32) {
+  cluster.sync();
+  if (part == 0 && threadIdx.x < 32) {
     Best b{-INFINITY, INT_MAX};
-    if (threadIdx.x < kArgmaxThreads / 32) b = Best{sv[threadIdx.x], si[threadIdx.x]};
+    if (threadIdx.x < kArgmaxSplit * kWarps) b = Best{sv[threadIdx.x], si[threadIdx.x]};
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
       Best o{__shfl_xor_sync(0xffffffffu, b.v, off), __shfl_xor_sync(0xffffffffu, b.i, off)};
@@ -91,8 +102,19 @@ argmax_rows_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
 int launch_argmax(const float* logits, int rows, int V, int64_t row_stride, int32_t* out,
                   cudaStream_t stream) {
   if (rows == 0) return SPECVLM_OK;
-  argmax_rows_kernel<<<rows, kArgmaxThreads, 0, stream>>>(logits, V, row_stride, out);
-  return check_cuda(cudaGetLastError(), "argmax launch");
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kArgmaxSplit, rows);
+  cfg.blockDim = dim3(kArgmaxThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kArgmaxSplit;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return check_cuda(cudaLaunchKernelEx(&cfg, argmax_rows_kernel, logits, V, row_stride, out), "argmax launch");
 }
 
 }  // namespace specvlm

@@ -5,6 +5,7 @@
 // with parent < child labels, its mask words, depths and position ids.
 #include "common.cuh"
 
+#include <limits.h>
 #include <math.h>
 
 namespace specvlm {
@@ -19,77 +20,63 @@ struct Cand {
 // larger value first; equal values: lower index first
 __device__ __forceinline__ bool before(const Cand& a, const Cand& b) { return a.v > b.v || (a.v == b.v && a.i < b.i); }
 
-// One block per logits row: every thread keeps the k best of its strided share in registers,
-// then k rounds of a block-wide tournament over the threads' current heads pick the row's top k
-// in order. The row's log-sum-exp comes from an online (max, sum) pass folded into the same scan.
-template <int K>
+// One block per logits row, k rounds. In every round each thread scans its strided share of the
+// row (served from L1/L2 after the first round) for its best element that comes strictly after
+// the previous round's winner in (value descending, index ascending) order, and a block-wide
+// reduction picks the round's winner. The first round also accumulates an online (max, sum) for
+// the row's log-sum-exp.
 __global__ void __launch_bounds__(kTopkThreads)
 topk_logprob_kernel(const float* __restrict__ logits, int V, int64_t row_stride, int k,
                     int32_t* __restrict__ tokens, float* __restrict__ logprob) {
   const int row = blockIdx.x;
   const float* x = logits + static_cast<int64_t>(row) * row_stride;
-  Cand best[K];
-#pragma unroll
-  for (int j = 0; j < K; ++j) best[j] = Cand{-INFINITY, INT_MAX};
-  float m = -INFINITY, z = 0.f;
-  for (int v = threadIdx.x; v < V; v += kTopkThreads) {
-    const float val = x[v];
-    if (val > m) { z = z * __expf(m - val) + 1.f; m = val; } else { z += __expf(val - m); }
-    Cand c{val, v};
-    if (before(c, best[K - 1])) {
-      best[K - 1] = c;
-#pragma unroll
-      for (int j = K - 1; j > 0; --j)
-        if (before(best[j], best[j - 1])) { const Cand t = best[j]; best[j] = best[j - 1]; best[j - 1] = t; }
-    }
-  }
   __shared__ float s_m[kTopkThreads / 32], s_z[kTopkThreads / 32];
   __shared__ Cand s_c[kTopkThreads / 32];
   __shared__ float s_lse;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // log-sum-exp: combine (max, sum) pairs
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    const float om = __shfl_xor_sync(0xffffffffu, m, off), oz = __shfl_xor_sync(0xffffffffu, z, off);
-    const float nm = fmaxf(m, om);
-    z = (m == -INFINITY ? 0.f : z * __expf(m - nm)) + (om == -INFINITY ? 0.f : oz * __expf(om - nm));
-    m = nm;
-  }
-  if (lane == 0) { s_m[warp] = m; s_z[warp] = z; }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float gm = -INFINITY, gz = 0.f;
-    for (int w = 0; w < kTopkThreads / 32; ++w) {
-      const float nm = fmaxf(gm, s_m[w]);
-      gz = (gm == -INFINITY ? 0.f : gz * __expf(gm - nm)) + (s_m[w] == -INFINITY ? 0.f : s_z[w] * __expf(s_m[w] - nm));
-      gm = nm;
-    }
-    s_lse = gm + logf(gz);
-  }
-  // tournament
-  int head = 0;
+  Cand last{INFINITY, -1};  // everything comes after it
   for (int r = 0; r < k; ++r) {
-    Cand c = Cand{-INFINITY, INT_MAX};
-#pragma unroll
-    for (int j = 0; j < K; ++j)
-      if (j == head) c = best[j];
+    Cand c{-INFINITY, INT_MAX};
+    float m = -INFINITY, z = 0.f;
+    for (int v = threadIdx.x; v < V; v += kTopkThreads) {
+      const float val = x[v];
+      const Cand e{val, v};
+      if (before(last, e) && before(e, c)) c = e;
+      if (r == 0) {
+        if (val > m) { z = z * __expf(m - val) + 1.f; m = val; } else { z += __expf(val - m); }
+      }
+    }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
       Cand o{__shfl_xor_sync(0xffffffffu, c.v, off), __shfl_xor_sync(0xffffffffu, c.i, off)};
       if (before(o, c)) c = o;
+      if (r == 0) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, off), oz = __shfl_xor_sync(0xffffffffu, z, off);
+        const float nm = fmaxf(m, om);
+        z = (m == -INFINITY ? 0.f : z * __expf(m - nm)) + (om == -INFINITY ? 0.f : oz * __expf(om - nm));
+        m = nm;
+      }
+    }
+    __syncthreads();  // s_c of the previous round has been read by everyone
+    if (lane == 0) {
+      s_c[warp] = c;
+      if (r == 0) { s_m[warp] = m; s_z[warp] = z; }
     }
     __syncthreads();
-    if (lane == 0) s_c[warp] = c;
-    __syncthreads();
     Cand w = s_c[0];
+#pragma unroll
     for (int q = 1; q < kTopkThreads / 32; ++q)
       if (before(s_c[q], w)) w = s_c[q];
-    // the thread that owns the winner advances; everyone knows the winner
-    bool mine = false;
-#pragma unroll
-    for (int j = 0; j < K; ++j)
-      if (j == head && best[j].i == w.i && w.i != INT_MAX) mine = true;
-    if (mine) ++head;
+    if (r == 0 && threadIdx.x == 0) {
+      float gm = -INFINITY, gz = 0.f;
+      for (int q = 0; q < kTopkThreads / 32; ++q) {
+        const float nm = fmaxf(gm, s_m[q]);
+        gz = (gm == -INFINITY ? 0.f : gz * __expf(gm - nm)) + (s_m[q] == -INFINITY ? 0.f : s_z[q] * __expf(s_m[q] - nm));
+        gm = nm;
+      }
+      s_lse = gm + logf(gz);
+    }
+    last = w;
     if (threadIdx.x == 0) {
       tokens[static_cast<int64_t>(row) * k + r] = (w.i == INT_MAX) ? 0 : w.i;
       logprob[static_cast<int64_t>(row) * k + r] = w.v - s_lse;
@@ -97,7 +84,7 @@ topk_logprob_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
   }
 }
 
-constexpr int kRerankThreads = 1024;
+constexpr int kRerankThreads = 1024;  // also the candidate limit
 
 // One block per sequence, one thread per candidate. Ranks come from counting: candidate i is
 // kept iff fewer than T-1 other candidates come before it in (score descending, index) order;
@@ -197,7 +184,7 @@ extern "C" int specvlm_topk_logprob(const float* logits, int rows, int V, int64_
   if (rows == 0) return SPECVLM_OK;
   SPECVLM_REQUIRE(logits && tokens && logprob, "topk_logprob: null pointer");
   SPECVLM_REQUIRE(row_stride >= V, "topk_logprob: row_stride must be >= V");
-  topk_logprob_kernel<kMaxK><<<rows, kTopkThreads, 0, static_cast<cudaStream_t>(stream)>>>(logits, V, row_stride, k,
+  topk_logprob_kernel<<<rows, kTopkThreads, 0, static_cast<cudaStream_t>(stream)>>>(logits, V, row_stride, k,
                                                                                         tokens, logprob);
   return check_cuda(cudaGetLastError(), "topk_logprob launch");
 }

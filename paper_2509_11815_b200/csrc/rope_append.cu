@@ -6,7 +6,7 @@
 // by position. A tree node's position is prefix length + depth, so siblings share a position.
 // Rotation: pairs (d, d + 64), angle = pos * base^(-2d/128), base 10000 by default.
 //
-// One block per (tree node, sequence). The 64 angles of the node are computed once: the product
+// One block per (tree node, sequence, group of heads). The 64 angles of the node are computed once: the product
 // pos * inv_freq and its reduction modulo 2 pi are done in double (positions reach 10^4, where a
 // float product would already be off by more than a bf16 step), sine and cosine in float. The
 // warps then loop over heads: q row -> rotated q, new k row -> rotated into cache slot P_b + t,
@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(kRopeThreads) rope_append_kernel(const RopePar
   // lane owns pairs d = 2*lane, 2*lane + 1 (elements d and d + 64)
   const float c0 = s_cos[2 * lane], s0 = s_sin[2 * lane], c1 = s_cos[2 * lane + 1], s1 = s_sin[2 * lane + 1];
   const int slot = p.prefix_len[b] + t;
-  for (int h = warp; h < p.H; h += kRopeThreads / 32) {
+  for (int h = blockIdx.z * (kRopeThreads / 32) + warp; h < p.H; h += gridDim.z * (kRopeThreads / 32)) {
     {
       const uint32_t* src = reinterpret_cast<const uint32_t*>(p.q_in + b * p.qi_sb + h * p.qi_sh + t * p.qi_st);
       uint32_t* dst = reinterpret_cast<uint32_t*>(p.q_out + b * p.qo_sb + h * p.qo_sh + t * p.qo_st);
@@ -141,7 +141,10 @@ extern "C" int specvlm_rope_append(const uint16_t* q_in, const uint16_t* k_new, 
   p.vc_sb = d->vc_stride_b; p.vc_sh = d->vc_stride_h; p.vc_ss = d->vc_stride_s;
   const double base = d->rope_base > 0.f ? static_cast<double>(d->rope_base) : 10000.0;
   for (int i = 0; i < 64; ++i) p.inv_freq[i] = pow(base, -2.0 * i / 128.0);
-  dim3 grid(d->T, d->B);
+  // enough blocks along z that a warp handles one or two heads
+  int gz = (d->H + 2 * (kRopeThreads / 32) - 1) / (2 * (kRopeThreads / 32));
+  if (static_cast<int64_t>(gz) * d->T * d->B > 4096) gz = 1;
+  dim3 grid(d->T, d->B, gz);
   rope_append_kernel<<<grid, kRopeThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
   return check_cuda(cudaGetLastError(), "rope_append launch");
 }
