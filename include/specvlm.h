@@ -337,6 +337,27 @@ SPECVLM_API int specvlm_accept_compact(const int32_t* draft_tokens, const int32_
                            int32_t* accept_len, int32_t* next_token, int32_t* new_prefix_len,
                            int32_t* status, void* stream);
 
+/*
+ * The whole verify step of an L-layer decoder in one host call (Sections 3.1, 3.2, 4.1): L
+ * attention launches (layer l uses q + l * q_stride_l, the layer-l slice of the caches and
+ * out + l * out_stride_l; q and out are [B][H][T][D] contiguous per layer), then
+ * specvlm_argmax over target_logits (fp32 [B][T][V] contiguous, V a multiple of 4), then
+ * specvlm_accept_compact over all layers. Arguments as in those calls; `workspace` is only
+ * needed when the attention call would need one (more than 8 KV splits).
+ * layers_independent != 0 declares that no layer's q / cache / out is written by the
+ * preceding layer's launch (e.g. precomputed or synthetic per-layer inputs): layers 1..L-1 are
+ * then launched with SPECVLM_ATTN_FLAG_INPUTS_STABLE and overlap. In a real decoder, where
+ * other kernels sit between the attention calls and feed them, call the per-layer entry points.
+ */
+SPECVLM_API int specvlm_verify_step(const uint16_t* q, int64_t q_stride_l, uint16_t* k_cache, uint16_t* v_cache,
+                        const specvlm_kv_desc* kv_desc_host, const int32_t* prefix_len,
+                        const int32_t* tree_parent, const uint64_t* tree_mask_bits,
+                        const int32_t* draft_tokens, const float* target_logits, int T, int V,
+                        uint16_t* out, int64_t out_stride_l, int32_t* argmax_tokens,
+                        int32_t* accepted_idx, int acc_stride, int32_t* accept_len,
+                        int32_t* next_token, int32_t* new_prefix_len, int layers_independent,
+                        void* workspace, int32_t* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -521,6 +521,8 @@ extern "C" int specvlm_tree_verify_attn(const uint16_t* q, const uint16_t* k_cac
 
   // Raising the dynamic shared memory limit is per function and per device.
   static bool attr_set[64] = {};
+  static std::mutex attr_mu;
+  std::lock_guard<std::mutex> attr_lock(attr_mu);
   int dev = 0;
   rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
   if (rc != SPECVLM_OK) return rc;

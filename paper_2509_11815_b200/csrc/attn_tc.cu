@@ -809,6 +809,8 @@ static int launch_cfg(const AttnParams& p, const specvlm_attn_desc& d, cudaStrea
   if (rc != SPECVLM_OK) return rc;
 
   static bool attr_set[64] = {};
+  static std::mutex attr_mu;
+  std::lock_guard<std::mutex> attr_lock(attr_mu);
   int dev = 0;
   rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
   if (rc != SPECVLM_OK) return rc;
