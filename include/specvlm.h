@@ -73,9 +73,10 @@ extern "C" {
  *   preceding kernel (true in a decoder layer, where the preceding kernel produces only q and
  *   the tree's own K/V rows): prefix tiles are prefetched early; q, the tree arrays and the
  *   tree slots are read only after the preceding kernel has completed.
- * INPUTS_STABLE: nothing this call reads is written by the preceding kernel, and `out` is
- *   neither read nor written by it: the whole call may overlap with it (back-to-back
- *   attention calls on independent inputs, as in a benchmark). */
+ * INPUTS_STABLE: nothing this call reads (q, caches, prefix_len, tree arrays) is written by the
+ *   preceding kernel: the whole call may overlap with it (back-to-back attention calls on
+ *   independent inputs, as in a benchmark). Its writes to `out` are still issued only after the
+ *   preceding kernel has completed. */
 #define SPECVLM_ATTN_FLAG_PREFIX_STABLE 2
 #define SPECVLM_ATTN_FLAG_INPUTS_STABLE 4
 /* Run in the configuration that occupies half an SM per thread block (chosen automatically for

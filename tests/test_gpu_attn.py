@@ -292,3 +292,49 @@ def test_invalid_arguments_are_rejected_on_the_host():
         flat = torch.empty(qt.numel() + 8, dtype=torch.bfloat16, device="cuda")
         q_bad = flat[1:1 + qt.numel()].view_as(qt)
         sv.specvlm_tree_verify_attn(q_bad, kt, vt, plt, None, mask_to_torch(masks), out, num_splits=1)
+
+
+@pytest.mark.parametrize("splits", [1, 2])
+def test_late_maximum_forces_the_accumulator_rescale(splits):
+    """Scores that jump by far more than 2^8 late in a CTA's key range: the output accumulator
+    has to be rescaled after earlier tiles were already accumulated."""
+    rng = np.random.default_rng(23)
+    H, T, P, D = 2, 26, 1500, 128
+    parent = wl.config1_tree(rng, T=T, max_depth=5)
+    mask = oracle.tree_mask_bits(parent)
+    qf = rng.standard_normal((1, H, T, D)).astype(np.float32)
+    kf = (0.05 * rng.standard_normal((1, H, P + T, D))).astype(np.float32)
+    for i in range(T):
+        # row i finds a key aligned with it deep in the prefix, a stronger one later, and (for
+        # even rows) the strongest one on its own tree slot, which is processed last
+        kf[0, :, 300 + 7 * i] = 1.5 * qf[0, :, i]
+        kf[0, :, 1100 + 5 * i] = 3.0 * qf[0, :, i]
+        if i % 2 == 0:
+            kf[0, :, P + i] = 6.0 * qf[0, :, i]
+    q, k = wl.bf16_bits_from_f32(qf), wl.bf16_bits_from_f32(kf)
+    v = wl.normal_bf16_bits(rng, (1, H, P + T, D))
+    ref = oracle_attn_all(q, k, v, [P], [mask])
+    got, status = run_attn(q, k, v, [P], masks=[mask], num_splits=splits)
+    assert status == 0
+    assert_attn_close(got, ref)
+    vf = oracle.bf16_bits_to_f64(v)
+    out = oracle.bf16_bits_to_f64(got)
+    for i in range(0, T, 2):     # even rows lock onto their own tree slot
+        assert np.abs(out[0, :, i] - vf[0, :, P + i]).max() < 2e-2
+
+
+def test_randomized_shape_sweep():
+    """Many random (batch, heads, tree size, ragged prefixes, split count) combinations."""
+    rng = np.random.default_rng(1234 + ATTN_FLAGS)
+    for trial in range(12):
+        B = int(rng.integers(1, 4))
+        H = int(rng.integers(1, 5))
+        T = int(rng.integers(1, 65))
+        prefixes = [int(x) for x in rng.integers(0, 900, size=B)]
+        splits = int(rng.choice([0, 1, 2, 3, 4, 6, 8, 11]))
+        q, k, v, pl, parents, masks = make_case(int(rng.integers(1 << 30)), B=B, H=H, T=T, prefixes=prefixes,
+                                                slack=int(rng.integers(0, 70)))
+        ref = oracle_attn_all(q, k, v, pl, masks)
+        got, status = run_attn(q, k, v, pl, masks=masks, num_splits=splits)
+        assert status == 0, (trial, B, H, T, prefixes, splits)
+        assert_attn_close(got, ref)
