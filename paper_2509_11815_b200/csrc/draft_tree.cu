@@ -20,11 +20,13 @@ struct Cand {
 // larger value first; equal values: lower index first
 __device__ __forceinline__ bool before(const Cand& a, const Cand& b) { return a.v > b.v || (a.v == b.v && a.i < b.i); }
 
-// One block per logits row, k rounds. In every round each thread scans its strided share of the
-// row (served from L1/L2 after the first round) for its best element that comes strictly after
-// the previous round's winner in (value descending, index ascending) order, and a block-wide
-// reduction picks the round's winner. The first round also accumulates an online (max, sum) for
-// the row's log-sum-exp.
+// One block per logits row. Every thread first loads its strided share of the row into registers
+// (up to 64 values, i.e. rows of up to 32768 entries; longer rows re-read global memory) and
+// accumulates an online (max, sum) for the row's log-sum-exp. Then k rounds: each thread finds its
+// best value that comes strictly after the previous round's winner in (value descending, index
+// ascending) order, and a block-wide reduction picks the round's winner.
+constexpr int kTopkRegs = 64;
+
 __global__ void __launch_bounds__(kTopkThreads)
 topk_logprob_kernel(const float* __restrict__ logits, int V, int64_t row_stride, int k,
                     int32_t* __restrict__ tokens, float* __restrict__ logprob) {
@@ -34,48 +36,73 @@ topk_logprob_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
   __shared__ Cand s_c[kTopkThreads / 32];
   __shared__ float s_lse;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const bool in_regs = V <= kTopkRegs * kTopkThreads;
+  float vals[kTopkRegs];
+  float m = -INFINITY, z = 0.f;
+#pragma unroll
+  for (int u = 0; u < kTopkRegs; ++u) {
+    const int v = threadIdx.x + u * kTopkThreads;
+    vals[u] = (in_regs && v < V) ? x[v] : -INFINITY;
+  }
+  if (in_regs) {
+#pragma unroll
+    for (int u = 0; u < kTopkRegs; ++u) m = fmaxf(m, vals[u]);
+#pragma unroll
+    for (int u = 0; u < kTopkRegs; ++u) z += (vals[u] == -INFINITY) ? 0.f : __expf(vals[u] - m);
+  } else {
+    for (int v = threadIdx.x; v < V; v += kTopkThreads) {
+      const float val = x[v];
+      if (val > m) { z = z * __expf(m - val) + 1.f; m = val; } else { z += __expf(val - m); }
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, off), oz = __shfl_xor_sync(0xffffffffu, z, off);
+    const float nm = fmaxf(m, om);
+    z = (m == -INFINITY ? 0.f : z * __expf(m - nm)) + (om == -INFINITY ? 0.f : oz * __expf(om - nm));
+    m = nm;
+  }
+  if (lane == 0) { s_m[warp] = m; s_z[warp] = z; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float gm = -INFINITY, gz = 0.f;
+    for (int q = 0; q < kTopkThreads / 32; ++q) {
+      const float nm = fmaxf(gm, s_m[q]);
+      gz = (gm == -INFINITY ? 0.f : gz * __expf(gm - nm)) + (s_m[q] == -INFINITY ? 0.f : s_z[q] * __expf(s_m[q] - nm));
+      gm = nm;
+    }
+    s_lse = gm + logf(gz);
+  }
   Cand last{INFINITY, -1};  // everything comes after it
   for (int r = 0; r < k; ++r) {
     Cand c{-INFINITY, INT_MAX};
-    float m = -INFINITY, z = 0.f;
-    for (int v = threadIdx.x; v < V; v += kTopkThreads) {
-      const float val = x[v];
-      const Cand e{val, v};
-      if (before(last, e) && before(e, c)) c = e;
-      if (r == 0) {
-        if (val > m) { z = z * __expf(m - val) + 1.f; m = val; } else { z += __expf(val - m); }
+    if (in_regs) {
+      // within a thread indices grow with u, so the first maximum in u order has the lowest index
+#pragma unroll
+      for (int u = 0; u < kTopkRegs; ++u) {
+        const int v = threadIdx.x + u * kTopkThreads;
+        const float val = vals[u];
+        const bool after = val < last.v || (val == last.v && v > last.i);
+        if (after && val > c.v && v < V) c = Cand{val, v};
+      }
+    } else {
+      for (int v = threadIdx.x; v < V; v += kTopkThreads) {
+        const Cand e{x[v], v};
+        if (before(last, e) && before(e, c)) c = e;
       }
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
       Cand o{__shfl_xor_sync(0xffffffffu, c.v, off), __shfl_xor_sync(0xffffffffu, c.i, off)};
       if (before(o, c)) c = o;
-      if (r == 0) {
-        const float om = __shfl_xor_sync(0xffffffffu, m, off), oz = __shfl_xor_sync(0xffffffffu, z, off);
-        const float nm = fmaxf(m, om);
-        z = (m == -INFINITY ? 0.f : z * __expf(m - nm)) + (om == -INFINITY ? 0.f : oz * __expf(om - nm));
-        m = nm;
-      }
     }
-    __syncthreads();  // s_c of the previous round has been read by everyone
-    if (lane == 0) {
-      s_c[warp] = c;
-      if (r == 0) { s_m[warp] = m; s_z[warp] = z; }
-    }
+    __syncthreads();  // s_c of the previous round (and s_lse) settled
+    if (lane == 0) s_c[warp] = c;
     __syncthreads();
     Cand w = s_c[0];
 #pragma unroll
     for (int q = 1; q < kTopkThreads / 32; ++q)
       if (before(s_c[q], w)) w = s_c[q];
-    if (r == 0 && threadIdx.x == 0) {
-      float gm = -INFINITY, gz = 0.f;
-      for (int q = 0; q < kTopkThreads / 32; ++q) {
-        const float nm = fmaxf(gm, s_m[q]);
-        gz = (gm == -INFINITY ? 0.f : gz * __expf(gm - nm)) + (s_m[q] == -INFINITY ? 0.f : s_z[q] * __expf(s_m[q] - nm));
-        gm = nm;
-      }
-      s_lse = gm + logf(gz);
-    }
     last = w;
     if (threadIdx.x == 0) {
       tokens[static_cast<int64_t>(row) * k + r] = (w.i == INT_MAX) ? 0 : w.i;
@@ -98,13 +125,13 @@ tree_rerank_kernel(const int32_t* __restrict__ cand_parent, const float* __restr
   const int b = blockIdx.x, i = threadIdx.x;
   cand_parent += static_cast<int64_t>(b) * C; cand_score += static_cast<int64_t>(b) * C;
   cand_token += static_cast<int64_t>(b) * C;
-  __shared__ float s_score[kRerankThreads];
+  __shared__ __align__(16) float s_score[kRerankThreads];
   __shared__ short s_par[kRerankThreads], s_depth[kRerankThreads], s_label[kRerankThreads];
   __shared__ int s_bad;
   __shared__ int s_tpar[SPECVLM_MAX_TREE];
   if (i == 0) s_bad = 0;
+  s_score[i] = (i < C) ? cand_score[i] : -INFINITY;
   if (i < C) {
-    s_score[i] = cand_score[i];
     const int p = cand_parent[i];
     s_par[i] = static_cast<short>(p);
     s_label[i] = -1;
@@ -127,21 +154,39 @@ tree_rerank_kernel(const int32_t* __restrict__ cand_parent, const float* __restr
     } else {
       const float si = s_score[i];
       int rank = 0;
-      for (int j = 1; j < C; ++j) {
-        const float sj = s_score[j];
-        rank += (sj > si || (sj == si && j < i)) ? 1 : 0;
+      // four scores per shared-memory load; entries at or beyond C were filled with -inf
+      const float4* sc4 = reinterpret_cast<const float4*>(s_score);
+      for (int j4 = 0; j4 < (C + 3) / 4; ++j4) {
+        const float4 sj = sc4[j4];
+        const int j = 4 * j4;
+        rank += (j > 0 && (sj.x > si || (sj.x == si && j < i))) ? 1 : 0;
+        rank += (sj.y > si || (sj.y == si && j + 1 < i)) ? 1 : 0;
+        rank += (sj.z > si || (sj.z == si && j + 2 < i)) ? 1 : 0;
+        rank += (sj.w > si || (sj.w == si && j + 3 < i)) ? 1 : 0;
       }
       keep = rank < T - 1;
     }
     s_label[i] = keep ? 0 : -1;
   }
   __syncthreads();
+  // compact list of the kept candidates, so that the relabelling only compares kept ones
+  __shared__ int s_nkept;
+  __shared__ short s_kept[SPECVLM_MAX_TREE];
+  if (i == 0) s_nkept = 0;
+  __syncthreads();
+  if (keep) {
+    const int slot = atomicAdd(&s_nkept, 1);
+    if (slot < SPECVLM_MAX_TREE) s_kept[slot] = static_cast<short>(i);
+  }
+  __syncthreads();
   int label = -1;
   if (keep) {
     const float si = s_score[i];
+    const int nk = min(s_nkept, SPECVLM_MAX_TREE);
     int cnt = 0;
-    for (int j = 0; j < C; ++j) {
-      if (j == i || s_label[j] < 0) continue;
+    for (int q = 0; q < nk; ++q) {
+      const int j = s_kept[q];
+      if (j == i) continue;
       const int dj = s_depth[j];
       const float sj = s_score[j];
       const bool first = (dj < depth) || (dj == depth && (sj > si || (sj == si && j < i)));
