@@ -9,8 +9,9 @@
 // cluster. A CTA uses less than half of an SM (about 105 KB of shared memory, 256 TMEM columns),
 // so the CTAs of the next launch can become resident while this launch drains.
 // Roles inside a CTA (192 threads):
-//   warp 0      TMA producer: Q once, then 64-key K tiles (ring of 3) and V tiles (ring of 2)
-//               with cp.async.bulk.tensor, 128-byte swizzle, no multicast; owns the TMEM allocation
+//   warp 0      TMA producer: Q once, then 64-key K tiles (ring of 3) and V tiles (ring of 2), one
+//               5-D cp.async.bulk.tensor per tile, 128-byte swizzle, no multicast; owns the TMEM
+//               allocation
 //   warp 1      one lane issues tcgen05.mma: S = Q K^T (M=64, N=64, K=16 x 8) into one of two TMEM
 //               buffers, O += P V (M=64, N=128, K=16 x 4); tcgen05.commit signals the mbarriers
 //   warps 2..5  softmax: tcgen05.ld of their 16 rows of S, tree mask as one 64-bit visibility word
@@ -115,11 +116,13 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
 }
 
 // ---- TMA
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
-                                            int c2, int c3) {
+// One copy brings both 64-column halves of `rows x 128` bf16 (coordinates: column 0, row, half 0,
+// head, sequence); the halves land one after the other, each as rows of 128 swizzled bytes.
+__device__ __forceinline__ void tma_load_rows(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row, int h,
+                                              int b) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %3, %5, %6}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(0), "r"(row), "r"(h), "r"(b)
       : "memory");
 }
 
@@ -320,22 +323,19 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
     if (lane == 0 && n_tiles > 0) {
       auto issue_q = [&]() {
         mbar_expect_tx(Q_FULL, kQBytes);
-        tma_load_4d(base + kOffQ, &map_q, Q_FULL, 0, 0, h, b);
-        tma_load_4d(base + kOffQ + kQBytes / 2, &map_q, Q_FULL, 64, 0, h, b);
+        tma_load_rows(base + kOffQ, &map_q, Q_FULL, 0, h, b);
       };
       auto issue_k = [&](int i) {
         const int sk = i % kKStages;
         const uint32_t dk = base + kOffK + sk * kKBytes;
         mbar_expect_tx(FULL_K(sk), kKBytes);
-        tma_load_4d(dk, &map_k, FULL_K(sk), 0, KEY0(i), h, b);
-        tma_load_4d(dk + kKBytes / 2, &map_k, FULL_K(sk), 64, KEY0(i), h, b);
+        tma_load_rows(dk, &map_k, FULL_K(sk), KEY0(i), h, b);
       };
       auto issue_v = [&](int i) {
         const int sv = i % kVStages;
         const uint32_t dv = base + kOffV + sv * kVBytes;
         mbar_expect_tx(FULL_V(sv), kVBytes);
-        tma_load_4d(dv, &map_v, FULL_V(sv), 0, KEY0(i), h, b);
-        tma_load_4d(dv + kVBytes / 2, &map_v, FULL_V(sv), 64, KEY0(i), h, b);
+        tma_load_rows(dv, &map_v, FULL_V(sv), KEY0(i), h, b);
         TRACE(8 + (i < 12 ? i : 12));
       };
       int ik = 0, iv = 0;
@@ -503,18 +503,27 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
       tc_fence_before();
       mbar_arrive(S_FREE(i & 1));
 
+      // tiles of prefix keys only (the common case) need no masking; the test is uniform over the CTA
+      if (key0 < 0 || key0 + kTile > P) {
+#pragma unroll
+        for (int hf = 0; hf < kHalves; ++hf) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const bool v = (((e & 2) ? vis1[hf] : vis0[hf]) >> (8 * j + (e & 1))) & 1ull;
+              s[hf][4 * j + e] = v ? s[hf][4 * j + e] : -INFINITY;
+            }
+          }
+        }
+      }
       float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
       for (int hf = 0; hf < kHalves; ++hf) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const bool v = (((e & 2) ? vis1[hf] : vis0[hf]) >> (8 * j + (e & 1))) & 1ull;
-            const float x = v ? s[hf][4 * j + e] : -INFINITY;
-            s[hf][4 * j + e] = x;
-            if (e & 2) mx1 = fmaxf(mx1, x); else mx0 = fmaxf(mx0, x);
-          }
+          mx0 = fmaxf(mx0, fmaxf(s[hf][4 * j + 0], s[hf][4 * j + 1]));
+          mx1 = fmaxf(mx1, fmaxf(s[hf][4 * j + 2], s[hf][4 * j + 3]));
         }
       }
       mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
@@ -778,18 +787,20 @@ EncodeFn encode_fn() {
   return fn;
 }
 
-// 4-D bf16 map over [dim3][dim2][rows][128] with element strides; box = 64 elements x box_rows rows.
+// 5-D bf16 map over [dim3][dim2][rows][2 halves][64] with element strides; box = 64 elements x
+// box_rows rows x both halves, so one copy fills a whole operand tile in the layout the 128-byte
+// swizzled matrix descriptors expect (half 0 rows, then half 1 rows).
 int make_map(CUtensorMap* map, const void* base, int rows, int dim2, int dim3, int64_t stride_row,
              int64_t stride2, int64_t stride3, int box_rows) {
-  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(tc::kD), static_cast<cuuint64_t>(rows),
-                              static_cast<cuuint64_t>(dim2), static_cast<cuuint64_t>(dim3)};
+  const cuuint64_t dims[5] = {64, static_cast<cuuint64_t>(rows), 2, static_cast<cuuint64_t>(dim2),
+                              static_cast<cuuint64_t>(dim3)};
   // a stride of 0 (size-1 dimension) is not accepted by the encoder: any positive multiple of 16 works there
   auto fix = [&](int64_t s, int64_t fallback) { return static_cast<cuuint64_t>((s > 0 ? s : fallback) * 2); };
-  const cuuint64_t strides[3] = {fix(stride_row, tc::kD), fix(stride2, static_cast<int64_t>(rows) * tc::kD),
+  const cuuint64_t strides[4] = {fix(stride_row, tc::kD), 128, fix(stride2, static_cast<int64_t>(rows) * tc::kD),
                                  fix(stride3, static_cast<int64_t>(rows) * tc::kD * dim2)};
-  const cuuint32_t box[4] = {64, static_cast<cuuint32_t>(box_rows), 1, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  CUresult r = encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+  const cuuint32_t box[5] = {64, static_cast<cuuint32_t>(box_rows), 2, 1, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box,
                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(SPECVLM_ERR_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string(r));
