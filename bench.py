@@ -281,7 +281,7 @@ def run_ours(args, cfg):
     desc_pipe0 = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0],
                                    flags=sv.ATTN_FLAG_PREFIX_STABLE | sv.ATTN_FLAG_HALF_SM)
     ws = sv.alloc_attn_workspace(desc_ser, dev)
-    launches_per_step = L + 2
+    launches_per_step = L + 3  # L attention launches, argmax, accept + compaction, tree_build
 
     def attn_layers(i, pipelined):
         par, drf, lg, mask = sets[i % N_INPUT_SETS]
@@ -295,6 +295,9 @@ def run_ours(args, cfg):
         sv.specvlm_argmax(lg, tok)
         sv.specvlm_accept_compact(drf, par, tok, k_cache, v_cache, prefix_len, acc_idx, acc_len, nxt, new_len,
                                   status)
+        # tree metadata (ancestor masks) of the tree that the next step verifies
+        par_n, _, _, mask_n = sets[(i + 1) % N_INPUT_SETS]
+        sv.specvlm_tree_build(par_n, prefix_len, mask_n, status=status)
 
     # The launches of one step are captured once per input set into CUDA graphs (the L
     # attention launches and the argmax + accept/compact tail separately, so that events
