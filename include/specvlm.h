@@ -303,6 +303,10 @@ SPECVLM_API int specvlm_accept(const int32_t* draft_tokens, const int32_t* tree_
  *   target_logits    fp32 [B][T][V] contiguous
  *   uniforms_accept  fp32 [B][T] in [0, 1): entry c is used for the keep test of node c
  *   uniforms_sample  fp32 [B][T] in [0, 1): entry u is used if the walk stops at node u
+ *   row_stats        fp32 [B][T][2] out, 8-byte aligned: for every node row, max of the logits and
+ *                    sum over the vocabulary of exp((logit - max) / temperature); computed by a
+ *                    first launch over all rows, read by the walk (so log p(x) of any token at any
+ *                    node is (logit - max) / temperature - log(sum))
  *   outputs as in specvlm_accept. fp32 arithmetic; a decision whose random number lies within
  *   rounding distance of its threshold may differ from an exact evaluation.
  */
@@ -310,7 +314,7 @@ SPECVLM_API int specvlm_accept_sample(const int32_t* draft_tokens, const int32_t
                           const float* target_logits, const float* uniforms_accept,
                           const float* uniforms_sample, float temperature, int B, int T, int V,
                           int32_t* accepted_idx, int acc_stride, int32_t* accept_len,
-                          int32_t* next_token, int32_t* status, void* stream);
+                          int32_t* next_token, float* row_stats, int32_t* status, void* stream);
 
 /*
  * KV compaction after acceptance (the KV cache is the resource the paper's cost model

@@ -122,7 +122,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.specvlm_accept.restype = i32
     lib.specvlm_accept.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, i32, vp, vp, vp, vp]
     lib.specvlm_accept_sample.restype = i32
-    lib.specvlm_accept_sample.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, i32, i32, i32, vp, i32, vp, vp, vp, vp]
+    lib.specvlm_accept_sample.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, i32, i32, i32, vp, i32, vp, vp, vp, vp,
+                                          vp]
     lib.specvlm_kv_compact.restype = i32
     lib.specvlm_kv_compact.argtypes = [vp, vp, ctypes.POINTER(KvDesc), vp, vp, i32, vp, vp, vp, vp]
     lib.specvlm_accept_compact.restype = i32
@@ -385,8 +386,10 @@ def specvlm_accept(draft_tokens: torch.Tensor, tree_parent: torch.Tensor, target
 def specvlm_accept_sample(draft_tokens: torch.Tensor, tree_parent: torch.Tensor, target_logits: torch.Tensor,
                           uniforms_accept: torch.Tensor, uniforms_sample: torch.Tensor, temperature: float,
                           accepted_idx: torch.Tensor, accept_len: torch.Tensor, next_token: torch.Tensor,
-                          status: Optional[torch.Tensor] = None) -> None:
-    """Temperature > 0 tree acceptance by speculative sampling; see include/specvlm.h."""
+                          row_stats: torch.Tensor, status: Optional[torch.Tensor] = None) -> None:
+    """Temperature > 0 tree acceptance by speculative sampling; see include/specvlm.h.
+
+    row_stats: float32 [B][T][2] output (row max, sum of exp((logit - max) / temperature))."""
     for name, t in (("draft_tokens", draft_tokens), ("tree_parent", tree_parent), ("accepted_idx", accepted_idx),
                     ("accept_len", accept_len), ("next_token", next_token)):
         _need(t, torch.int32, name)
@@ -396,10 +399,13 @@ def specvlm_accept_sample(draft_tokens: torch.Tensor, tree_parent: torch.Tensor,
         if not t.is_contiguous():
             raise SpecvlmError(f"{name} must be contiguous")
     B, T = draft_tokens.shape
+    _need(row_stats, torch.float32, "row_stats")
+    if not row_stats.is_contiguous() or row_stats.numel() != B * T * 2:
+        raise SpecvlmError("row_stats must be a contiguous float32 tensor of B * T * 2 elements")
     _check(load_library().specvlm_accept_sample(
         _ptr(draft_tokens), _ptr(tree_parent), _ptr(target_logits), _ptr(uniforms_accept), _ptr(uniforms_sample),
         float(temperature), B, T, target_logits.shape[-1], _ptr(accepted_idx), accepted_idx.shape[1],
-        _ptr(accept_len), _ptr(next_token), _ptr(status), _stream()))
+        _ptr(accept_len), _ptr(next_token), _ptr(row_stats), _ptr(status), _stream()))
 
 
 def make_kv_desc(cache: torch.Tensor) -> KvDesc:

@@ -40,8 +40,8 @@ argmax_rows_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
                    int32_t* __restrict__ out) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
-  const int row = blockIdx.y;
-  const int part = blockIdx.x;  // == rank in the cluster
+  const int row = blockIdx.x / kArgmaxSplit;
+  const int part = blockIdx.x % kArgmaxSplit;  // == rank in the cluster
   const float* x = logits + static_cast<int64_t>(row) * row_stride;
   const float4* x4 = reinterpret_cast<const float4*>(x);
   const int n4 = V >> 2;
@@ -103,7 +103,7 @@ int launch_argmax(const float* logits, int rows, int V, int64_t row_stride, int3
                   cudaStream_t stream) {
   if (rows == 0) return SPECVLM_OK;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(kArgmaxSplit, rows);
+  cfg.gridDim = dim3(static_cast<unsigned>(kArgmaxSplit) * rows);  // rows along x: no 65535 limit
   cfg.blockDim = dim3(kArgmaxThreads);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;

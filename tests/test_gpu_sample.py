@@ -17,12 +17,21 @@ def gpu_accept_sample(parents, drafts, logits, ua, us, temperature, acc_stride=8
     idx = torch.full((B, acc_stride), -99, **i32)
     n, nxt = torch.full((B,), -99, **i32), torch.full((B,), -99, **i32)
     status = torch.zeros(1, **i32)
+    stats = torch.full((B, T, 2), float("nan"), dtype=torch.float32, device="cuda")
     sv.specvlm_accept_sample(torch.tensor(drafts, **i32), torch.tensor(parents, **i32),
                              torch.from_numpy(np.ascontiguousarray(logits, dtype=np.float32)).cuda(),
                              torch.from_numpy(np.ascontiguousarray(ua, dtype=np.float32)).cuda(),
                              torch.from_numpy(np.ascontiguousarray(us, dtype=np.float32)).cuda(),
-                             temperature, idx, n, nxt, status)
+                             temperature, idx, n, nxt, stats, status)
     torch.cuda.synchronize()
+    # the row statistics are an output too: max bit-exact, partition sum = 1 / (largest probability)
+    lg64 = np.asarray(logits, dtype=np.float64)
+    got = stats.cpu().numpy()
+    for b in range(min(B, 16)):
+        for t in range(0, T, 7):
+            p = oracle.softmax_f64(lg64[b, t], temperature)
+            assert got[b, t, 0] == np.float32(lg64[b, t].max())
+            assert abs(got[b, t, 1] * p.max() - 1.0) < 2e-5, (b, t, got[b, t, 1], 1.0 / p.max())
     return idx.cpu().numpy(), n.cpu().numpy(), nxt.cpu().numpy(), status.item()
 
 
@@ -37,7 +46,8 @@ def draw_robust_uniforms(rng, parent, draft, logits, temperature, margin):
     raise AssertionError("could not draw robust uniforms")
 
 
-@pytest.mark.parametrize("V,temperature,scale", [(32000, 1.0, 3.0), (32000, 0.7, 2.0), (1000, 1.0, 1.0), (17, 1.3, 1.0)])
+@pytest.mark.parametrize("V,temperature,scale", [(32000, 1.0, 3.0), (32000, 0.7, 2.0), (1000, 1.0, 1.0), (17, 1.3, 1.0), (40000, 1.0, 3.0),
+                                                 (32768, 0.8, 2.0), (1026, 1.0, 2.0)])
 def test_accept_sample_matches_oracle_on_robust_draws(V, temperature, scale):
     rng = np.random.default_rng(V)
     B, T = 12, 60
