@@ -5,6 +5,7 @@
 // with parent < child labels, its mask words, depths and position ids.
 #include "common.cuh"
 
+#include <cooperative_groups.h>
 #include <limits.h>
 #include <math.h>
 
@@ -52,7 +53,7 @@ topk_logprob_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
   } else {
     for (int v = threadIdx.x; v < V; v += kTopkThreads) {
       const float val = x[v];
-      if (val > m) { z = z * __expf(m - val) + 1.f; m = val; } else { z += __expf(val - m); }
+      if (val > m) { z = z * __expf(m - val) + 1.f; m = val; } else if (val > -INFINITY) { z += __expf(val - m); }
     }
   }
 #pragma unroll
@@ -107,6 +108,191 @@ topk_logprob_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
     if (threadIdx.x == 0) {
       tokens[static_cast<int64_t>(row) * k + r] = (w.i == INT_MAX) ? 0 : w.i;
       logprob[static_cast<int64_t>(row) * k + r] = w.v - s_lse;
+    }
+  }
+}
+
+// ---- cluster version: the row is shared by eight thread blocks
+//
+// One cluster of kTkSplit blocks per logits row. Every thread keeps kU groups of four consecutive
+// logits in registers (one 16-byte load each, all in flight together). Each block computes the
+// (max, sum) pair and the sorted top k of its share with k selection rounds over registers; the
+// lists and pairs meet in the first block's shared memory through distributed shared memory,
+// where the final order is found by counting: a candidate's position is the number of candidates
+// that come before it in (value descending, index ascending) order.
+constexpr int kTkThreads = 256;
+constexpr int kTkSplit = 8;
+
+// Unsigned key whose integer order is the order of the floats (-0 counted as +0).
+__device__ __forceinline__ unsigned ordered_key(float v) {
+  const unsigned u = __float_as_uint(v + 0.f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_value(unsigned key) {
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
+// Entries of exhausted lists carry value -inf and an index at or above kSentinel0, made unique
+// by the writer, so that (value descending, index ascending) orders all entries strictly.
+constexpr int kSentinel0 = INT_MAX - 4096;
+
+// Position of entry `me` among kLists sorted lists of k entries stored kMaxK apart: the number of
+// entries that come before it = the sum of its lower bounds in every list (its own place in its
+// own list). The binary searches of different lists are independent of one another.
+template <int kLists>
+__device__ __forceinline__ int rank_among(const Cand* lists, int k, const Cand me) {
+  int rank = 0;
+#pragma unroll
+  for (int l = 0; l < kLists; ++l) {
+    int lo = 0, hi = k;
+#pragma unroll
+    for (int step = 0; step < 5; ++step) {  // k <= 16 < 2^5
+      if (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (before(lists[l * kMaxK + mid], me)) lo = mid + 1; else hi = mid;
+      }
+    }
+    rank += lo;
+  }
+  return rank;
+}
+
+template <int kU>
+__global__ void __launch_bounds__(kTkThreads)
+topk_cluster_kernel(const float* __restrict__ logits, int V, int64_t row_stride, int k, int vec,
+                    int32_t* __restrict__ tokens, float* __restrict__ logprob) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int row = blockIdx.x / kTkSplit, part = blockIdx.x % kTkSplit;  // part == rank in the cluster
+  const float* x = logits + static_cast<int64_t>(row) * row_stride;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int kWarps = kTkThreads / 32;
+  __shared__ float s_m[kWarps], s_z[kWarps];
+  __shared__ Cand s_all[kTkSplit * kMaxK];  // used in the first block: every block's sorted list
+  __shared__ float s_pm[kTkSplit], s_pz[kTkSplit];
+  cluster.barrier_arrive();  // matched by the wait before the first remote store
+
+  const int n4 = (V + 3) >> 2;
+  const int per = (n4 + kTkSplit - 1) / kTkSplit;  // host guarantees per <= kU * kTkThreads
+  const int g0 = part * per, g1 = min(g0 + per, n4);
+  float vals[kU * 4];
+#pragma unroll
+  for (int u = 0; u < kU; ++u) {
+    const int g = g0 + u * kTkThreads + threadIdx.x;
+    float4 t = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    if (g < g1) {
+      if (vec) {
+        t = __ldg(reinterpret_cast<const float4*>(x) + g);
+      } else {
+        const int v = g << 2;
+        t.x = x[v];
+        if (v + 1 < V) t.y = x[v + 1];
+        if (v + 2 < V) t.z = x[v + 2];
+        if (v + 3 < V) t.w = x[v + 3];
+      }
+    }
+    vals[4 * u] = t.x; vals[4 * u + 1] = t.y; vals[4 * u + 2] = t.z; vals[4 * u + 3] = t.w;
+  }
+  // element e of group u is logit index 4 * (g0 + u * kTkThreads + threadIdx.x) + e: increasing in (u, e)
+  const int vbase = (g0 + static_cast<int>(threadIdx.x)) << 2;
+
+  float m = -INFINITY, z = 0.f;
+#pragma unroll
+  for (int i = 0; i < kU * 4; ++i) m = fmaxf(m, vals[i]);
+#pragma unroll
+  for (int i = 0; i < kU * 4; ++i) z += (vals[i] == -INFINITY) ? 0.f : __expf(vals[i] - m);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, off), oz = __shfl_xor_sync(0xffffffffu, z, off);
+    const float nm = fmaxf(m, om);
+    z = (m == -INFINITY ? 0.f : z * __expf(m - nm)) + (om == -INFINITY ? 0.f : oz * __expf(om - nm));
+    m = nm;
+  }
+  if (lane == 0) { s_m[warp] = m; s_z[warp] = z; }
+
+  // ---- k selection rounds inside every warp, no block-wide step: each round's winner is the best
+  // entry of the warp that comes strictly after the previous winner, found with two warp-wide
+  // integer reductions (largest order-preserving key, then lowest index among its holders);
+  // lane r keeps the winner of round r
+  Cand last{INFINITY, -1};
+  Cand kept{-INFINITY, INT_MAX};
+  for (int r = 0; r < k; ++r) {
+    Cand c{-INFINITY, INT_MAX};
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int v = vbase + u * (kTkThreads * 4) + e;
+        const float val = vals[4 * u + e];
+        const bool after = val < last.v || (val == last.v && v > last.i);
+        if (after && val > c.v) c = Cand{val, v};  // first maximum in (u, e) order = lowest index
+      }
+    }
+    const unsigned key = ordered_key(c.v);
+    const unsigned kmax = __reduce_max_sync(0xffffffffu, key);
+    const unsigned imin = __reduce_min_sync(0xffffffffu, key == kmax ? static_cast<unsigned>(c.i) : 0xffffffffu);
+    // an exhausted warp reduces to (-inf, INT_MAX): INT_MAX is the smallest index any lane reports then
+    const Cand w{key_value(kmax), static_cast<int>(imin)};
+    last = w;
+    if (lane == r) kept = w;
+  }
+  if (kept.i == INT_MAX) kept.i = kSentinel0 + (part * kWarps + warp) * kMaxK + lane;  // unique per entry
+  // ---- the warps' sorted lists are merged by counting
+  __shared__ Cand s_wl[kWarps * kMaxK];
+  __shared__ Cand s_top[kMaxK];
+  if (lane < k) s_wl[warp * kMaxK + lane] = kept;
+  __syncthreads();
+  // Two threads per entry (entry = list * kMaxK + place), each searching half of the lists: with a
+  // single warp per scheduler a chain of dependent instructions issues once every few cycles, so
+  // the work is spread over all warps of the block.
+  static_assert(kWarps == 8 && kTkSplit == 8 && kTkThreads == 2 * 8 * kMaxK, "merge layout");
+  __shared__ int s_part[2][8 * kMaxK];
+  const int entry = threadIdx.x & (8 * kMaxK - 1), half = threadIdx.x >> 7;
+  const bool live = (entry % kMaxK) < k;
+  {
+    const Cand me = s_wl[entry];
+    s_part[half][entry] = live ? rank_among<4>(s_wl + half * 4 * kMaxK, k, me) : 0;
+    __syncthreads();
+    const int rank = s_part[0][entry] + s_part[1][entry];
+    if (half == 0 && live && rank < k) s_top[rank] = me;
+  }
+  __syncthreads();
+  if (static_cast<int>(threadIdx.x) < k) kept = s_top[threadIdx.x];
+
+  // ---- lists and (max, sum) pairs meet in the first block
+  cluster.barrier_wait();
+  if (static_cast<int>(threadIdx.x) < k) cluster.map_shared_rank(s_all, 0)[part * kMaxK + threadIdx.x] = kept;
+  if (threadIdx.x == 0) {
+    float gm = -INFINITY, gz = 0.f;
+    for (int q = 0; q < kWarps; ++q) {
+      const float nm = fmaxf(gm, s_m[q]);
+      gz = (gm == -INFINITY ? 0.f : gz * __expf(gm - nm)) + (s_m[q] == -INFINITY ? 0.f : s_z[q] * __expf(s_m[q] - nm));
+      gm = nm;
+    }
+    cluster.map_shared_rank(s_pm, 0)[part] = gm;
+    cluster.map_shared_rank(s_pz, 0)[part] = gz;
+  }
+  cluster.sync();
+  if (part != 0) return;
+  __shared__ float s_lse;
+  if (threadIdx.x == 0) {
+    float gm = -INFINITY, gz = 0.f;
+    for (int q = 0; q < kTkSplit; ++q) {
+      const float nm = fmaxf(gm, s_pm[q]);
+      gz = (gm == -INFINITY ? 0.f : gz * __expf(gm - nm)) + (s_pm[q] == -INFINITY ? 0.f : s_pz[q] * __expf(s_pm[q] - nm));
+      gm = nm;
+    }
+    s_lse = gm + logf(gz);
+  }
+  __syncthreads();
+  {
+    const Cand me = s_all[entry];
+    s_part[half][entry] = live ? rank_among<4>(s_all + half * 4 * kMaxK, k, me) : 0;
+    __syncthreads();
+    const int rank = s_part[0][entry] + s_part[1][entry];
+    if (half == 0 && live && rank < k) {
+      tokens[static_cast<int64_t>(row) * k + rank] = (me.i >= kSentinel0) ? 0 : me.i;
+      logprob[static_cast<int64_t>(row) * k + rank] = me.v - s_lse;
     }
   }
 }
@@ -229,6 +415,33 @@ extern "C" int specvlm_topk_logprob(const float* logits, int rows, int V, int64_
   if (rows == 0) return SPECVLM_OK;
   SPECVLM_REQUIRE(logits && tokens && logprob, "topk_logprob: null pointer");
   SPECVLM_REQUIRE(row_stride >= V, "topk_logprob: row_stride must be >= V");
+  const int n4 = (V + 3) / 4;
+  const int per = (n4 + kTkSplit - 1) / kTkSplit;  // 16-byte groups per block of the cluster
+  if (per <= 32 * kTkThreads) {
+    const int vec = (V % 4 == 0) && (row_stride % 4 == 0) && aligned16(logits);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(kTkSplit) * rows);
+    cfg.blockDim = dim3(kTkThreads);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kTkSplit;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+    if (per <= 4 * kTkThreads)  // rows of up to 32768 logits
+      e = cudaLaunchKernelEx(&cfg, topk_cluster_kernel<4>, logits, V, row_stride, k, vec, tokens, logprob);
+    else if (per <= 8 * kTkThreads)
+      e = cudaLaunchKernelEx(&cfg, topk_cluster_kernel<8>, logits, V, row_stride, k, vec, tokens, logprob);
+    else if (per <= 16 * kTkThreads)
+      e = cudaLaunchKernelEx(&cfg, topk_cluster_kernel<16>, logits, V, row_stride, k, vec, tokens, logprob);
+    else  // up to 262144
+      e = cudaLaunchKernelEx(&cfg, topk_cluster_kernel<32>, logits, V, row_stride, k, vec, tokens, logprob);
+    return check_cuda(e, "topk_logprob launch");
+  }
+  // longer rows: one block per row, re-reading global memory in every round
   topk_logprob_kernel<<<rows, kTopkThreads, 0, static_cast<cudaStream_t>(stream)>>>(logits, V, row_stride, k,
                                                                                         tokens, logprob);
   return check_cuda(cudaGetLastError(), "topk_logprob launch");

@@ -82,6 +82,13 @@ def test_argmax_matches_oracle_bit_exact(V):
     assert np.array_equal(got, oracle.vocab_argmax(x))
 
 
+def test_argmax_more_rows_than_one_grid_dimension_holds():
+    """B * T > 65535 rows: rows are laid along grid x, which has no such limit."""
+    rng = np.random.default_rng(65536)
+    x = rng.standard_normal((1100, 60, 64), dtype=np.float32)
+    assert np.array_equal(gpu_argmax(x), oracle.vocab_argmax(x))
+
+
 def test_argmax_tie_rules():
     V = 32000
     rng = np.random.default_rng(3)

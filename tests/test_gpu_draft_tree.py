@@ -10,15 +10,24 @@ import paper_2509_11815_b200 as sv
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("V,k", [(32000, 10), (32001, 16), (50, 10), (16, 16), (1000, 1)])
-def test_topk_logprob_matches_oracle(V, k):
+@pytest.mark.parametrize("V,k,pad", [(32000, 10, 0), (32001, 16, 0), (50, 10, 0), (16, 16, 0), (1000, 1, 0),
+                                     (32000, 10, 8), (32000, 7, 3), (40000, 10, 0), (100003, 5, 0),
+                                     (151936, 10, 0), (300000, 4, 0)])
+def test_topk_logprob_matches_oracle(V, k, pad):
+    """Rows of every length class (register-resident shares of 16 to 128 values per thread, and the
+    one-block-per-row kernel beyond 262144), aligned and unaligned row strides."""
     rng = np.random.default_rng(V + k)
     rows = 13
     x = (rng.standard_normal((rows, V)) * 2).astype(np.float32)
     x[0, V // 3] = x[0, V // 2] = x[0].max() + 1.0          # equal maxima: lower id first
     x[1, :] = 0.5                                           # constant row: ids 0..k-1
     x[2, V - 1] = 50.0                                      # a dominant last token
-    lg = torch.from_numpy(x).cuda()
+    if V >= 1000:
+        x[3, 1::2] = -np.inf                                # masked vocabulary entries never win
+        x[4, : V - 40] = -np.inf                            # everything finite sits in the last block's share
+    store = torch.full((rows, V + pad), 1e30, dtype=torch.float32, device="cuda")   # padding must never win
+    store[:, :V] = torch.from_numpy(x).cuda()
+    lg = store[:, :V]
     toks = torch.full((rows, k), -1, dtype=torch.int32, device="cuda")
     lps = torch.zeros((rows, k), dtype=torch.float32, device="cuda")
     sv.specvlm_topk_logprob(lg, k, toks, lps)
