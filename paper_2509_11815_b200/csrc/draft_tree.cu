@@ -299,9 +299,10 @@ topk_cluster_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
 
 constexpr int kRerankThreads = 1024;  // also the candidate limit
 
-// One block per sequence, one thread per candidate. Ranks come from counting: candidate i is
-// kept iff fewer than T-1 other candidates come before it in (score descending, index) order;
-// its new label is the number of kept candidates before it in (depth, score descending, index).
+// One block per sequence, one thread per candidate. A candidate is kept iff it is the root or
+// among the T - 1 best others in (score descending, index ascending) order, decided by a radix
+// select on unique keys; its new label is the number of kept candidates before it in (depth,
+// score descending, index ascending) order, counted with warp ballots over the kept list.
 __global__ void __launch_bounds__(kRerankThreads)
 tree_rerank_kernel(const int32_t* __restrict__ cand_parent, const float* __restrict__ cand_score,
                    const int32_t* __restrict__ cand_token, const int32_t* __restrict__ prefix_len, int C, int T,
@@ -312,7 +313,7 @@ tree_rerank_kernel(const int32_t* __restrict__ cand_parent, const float* __restr
   cand_parent += static_cast<int64_t>(b) * C; cand_score += static_cast<int64_t>(b) * C;
   cand_token += static_cast<int64_t>(b) * C;
   __shared__ __align__(16) float s_score[kRerankThreads];
-  __shared__ short s_par[kRerankThreads], s_depth[kRerankThreads], s_label[kRerankThreads];
+  __shared__ short s_par[kRerankThreads], s_label[kRerankThreads];
   __shared__ int s_bad;
   __shared__ int s_tpar[SPECVLM_MAX_TREE];
   if (i == 0) s_bad = 0;
@@ -331,55 +332,106 @@ tree_rerank_kernel(const int32_t* __restrict__ cand_parent, const float* __restr
   }
   __syncthreads();
   const bool bad = s_bad != 0;
+  // ---- which candidates stay: the root and the T - 1 best of the others in (score descending,
+  // index ascending) order. Every candidate gets a unique 48-bit key (order-preserving score
+  // bits, then 65535 - index); a radix select over six 8-bit digits finds the key of the
+  // (T - 1)-th largest, and a candidate stays iff its key is not below it.
+  __shared__ int s_hist[256], s_wsum[8], s_digit, s_remaining;
+  unsigned long long key = 0ull;
   if (i < C && !bad) {
     int n = i;
     while (n > 0) { n = s_par[n]; ++depth; }
-    s_depth[i] = static_cast<short>(depth);
-    if (i == 0) {
-      keep = true;
-    } else {
-      const float si = s_score[i];
-      int rank = 0;
-      // four scores per shared-memory load; entries at or beyond C were filled with -inf
-      const float4* sc4 = reinterpret_cast<const float4*>(s_score);
-      for (int j4 = 0; j4 < (C + 3) / 4; ++j4) {
-        const float4 sj = sc4[j4];
-        const int j = 4 * j4;
-        rank += (j > 0 && (sj.x > si || (sj.x == si && j < i))) ? 1 : 0;
-        rank += (sj.y > si || (sj.y == si && j + 1 < i)) ? 1 : 0;
-        rank += (sj.z > si || (sj.z == si && j + 2 < i)) ? 1 : 0;
-        rank += (sj.w > si || (sj.w == si && j + 3 < i)) ? 1 : 0;
+    if (i > 0) key = (static_cast<unsigned long long>(ordered_key(s_score[i])) << 16) | static_cast<unsigned>(65535 - i);
+  }
+  bool active = i > 0 && i < C && !bad;
+  int remaining = T - 1;  // the wanted key is the remaining-th largest among the active ones
+  unsigned long long threshold = 0ull;
+  if (T > 1) {
+#pragma unroll 1
+    for (int shift = 40; shift >= 0; shift -= 8) {
+      if (i < 256) s_hist[i] = 0;
+      __syncthreads();
+      const int digit = static_cast<int>((key >> shift) & 0xffull);
+      if (active) atomicAdd(&s_hist[digit], 1);
+      __syncthreads();
+      // suffix sums over the 256 bins: above[d] = number of active keys with a larger digit
+      int h = 0, incl = 0;
+      if (i < 256) {
+        h = s_hist[255 - i];  // thread i looks at digit 255 - i, so a forward scan is a suffix sum
+        incl = h;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int o = __shfl_up_sync(0xffffffffu, incl, off);
+          if ((i & 31) >= off) incl += o;
+        }
+        if ((i & 31) == 31) s_wsum[i >> 5] = incl;
       }
-      keep = rank < T - 1;
+      __syncthreads();
+      if (i < 256) {
+        for (int w = 0; w < (i >> 5); ++w) incl += s_wsum[w];
+        const int above = incl - h;
+        if (above < remaining && incl >= remaining) {  // exactly one digit satisfies this
+          s_digit = 255 - i;
+          s_remaining = remaining - above;
+        }
+      }
+      __syncthreads();
+      const int d = s_digit;
+      remaining = s_remaining;
+      threshold |= static_cast<unsigned long long>(d) << shift;
+      active = active && digit == d;
     }
+  }
+  if (i < C && !bad) {
+    keep = i == 0 || (T > 1 && key >= threshold);
     s_label[i] = keep ? 0 : -1;
   }
   __syncthreads();
-  // compact list of the kept candidates, so that the relabelling only compares kept ones
+  // ---- compact list of the kept candidates (any order), then labels by counting among them:
+  // warp w ranks list slots 2 w and 2 w + 1, one ballot per 32 list entries
   __shared__ int s_nkept;
-  __shared__ short s_kept[SPECVLM_MAX_TREE];
+  __shared__ short s_kept[SPECVLM_MAX_TREE], s_kdepth[SPECVLM_MAX_TREE], s_klabel[SPECVLM_MAX_TREE];
+  __shared__ float s_kscore[SPECVLM_MAX_TREE];
   if (i == 0) s_nkept = 0;
   __syncthreads();
+  int my_slot = -1;
   if (keep) {
-    const int slot = atomicAdd(&s_nkept, 1);
-    if (slot < SPECVLM_MAX_TREE) s_kept[slot] = static_cast<short>(i);
+    my_slot = atomicAdd(&s_nkept, 1);
+    if (my_slot < SPECVLM_MAX_TREE) {
+      s_kept[my_slot] = static_cast<short>(i);
+      s_kdepth[my_slot] = static_cast<short>(depth);
+      s_kscore[my_slot] = s_score[i];
+    }
+  }
+  __syncthreads();
+  {
+    const int nk = min(s_nkept, SPECVLM_MAX_TREE);
+    const int lane = i & 31, warp = i >> 5;
+#pragma unroll
+    for (int sub = 0; sub < 2; ++sub) {
+      const int m = 2 * warp + sub;  // warp-uniform
+      if (m < nk) {
+        const int mi = s_kept[m], md = s_kdepth[m];
+        const float ms = s_kscore[m];
+        int cnt = 0;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int q = lane + 32 * half;
+          bool first = false;
+          if (q < nk && q != m) {
+            const int qi = s_kept[q], qd = s_kdepth[q];
+            const float qs = s_kscore[q];
+            first = (qd < md) || (qd == md && (qs > ms || (qs == ms && qi < mi)));
+          }
+          cnt += __popc(__ballot_sync(0xffffffffu, first));
+        }
+        if (lane == 0) s_klabel[m] = static_cast<short>(cnt);
+      }
+    }
   }
   __syncthreads();
   int label = -1;
-  if (keep) {
-    const float si = s_score[i];
-    const int nk = min(s_nkept, SPECVLM_MAX_TREE);
-    int cnt = 0;
-    for (int q = 0; q < nk; ++q) {
-      const int j = s_kept[q];
-      if (j == i) continue;
-      const int dj = s_depth[j];
-      const float sj = s_score[j];
-      const bool first = (dj < depth) || (dj == depth && (sj > si || (sj == si && j < i)));
-      cnt += first ? 1 : 0;
-    }
-    label = cnt;
-  }
+  if (keep && my_slot < SPECVLM_MAX_TREE) label = s_klabel[my_slot];
   __syncthreads();
   if (keep) s_label[i] = static_cast<short>(label);
   __syncthreads();

@@ -94,3 +94,37 @@ def test_tree_rerank_flags_scores_that_increase_along_a_path_and_bad_arguments()
     assert status.item() & sv.STATUS_BAD_TREE
     with pytest.raises(sv.SpecvlmError):
         sv.specvlm_tree_rerank(cp, cs, ct, 5, tp, dt)           # T > C
+
+
+@pytest.mark.parametrize("C,T", [(1024, 64), (64, 64), (300, 33), (5, 1), (2, 2)])
+def test_tree_rerank_many_exact_ties_and_extreme_sizes(C, T):
+    """Scores on a coarse grid (many exactly equal, signed zeros included), so the index part of the
+    order decides most of the selection; the candidate limit, C == T and T == 1."""
+    rng = np.random.default_rng(C * 100 + T)
+    B = 5
+    cps, css, cts = [], [], []
+    for b in range(B):
+        parent = np.full(C, -1, dtype=np.int32)
+        score = np.zeros(C, dtype=np.float32)
+        for c in range(1, C):
+            parent[c] = int(rng.integers(max(0, c - 40), c))
+            step = float(rng.integers(0, 3)) * 0.25          # 0 keeps the parent's score exactly
+            score[c] = np.float32(score[parent[c]] - step)
+        if b == 1:
+            score[score == 0] = np.float32(-0.0)             # -0 and +0 compare equal
+            score[0] = np.float32(0.0)
+        cps.append(parent), css.append(score), cts.append(rng.integers(0, 32000, size=C).astype(np.int32))
+    i32 = dict(dtype=torch.int32, device="cuda")
+    cp, ct = torch.tensor(np.stack(cps), **i32), torch.tensor(np.stack(cts), **i32)
+    cs = torch.tensor(np.stack(css), dtype=torch.float32, device="cuda")
+    tp, dt, kept = (torch.full((B, T), -9, **i32) for _ in range(3))
+    mask = torch.zeros((B, T), dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, **i32)
+    sv.specvlm_tree_rerank(cp, cs, ct, T, tp, dt, kept, mask, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    for b in range(B):
+        parent, tokens, kept_ids = oracle.rerank_tree(cps[b], css[b], cts[b], T)
+        assert np.array_equal(kept[b].cpu().numpy(), kept_ids)
+        assert np.array_equal(tp[b].cpu().numpy(), parent) and np.array_equal(dt[b].cpu().numpy(), tokens)
+        assert np.array_equal(mask[b].cpu().numpy().view(np.uint64), oracle.tree_mask_bits(parent))
