@@ -225,6 +225,82 @@ def workload_config(cfg):
 # ----------------------------------------------------------------------------- GPU arm
 
 
+def time_widened_rows(sv, cfg, dev):
+    """Microseconds per launch of the kernels next to the verify step (positioned inputs, temperature > 0
+    acceptance, draft-tree construction, parameter-free visual compression) at this workload's shapes.
+    Each kernel is replayed from a CUDA graph of 24 launches that rotate over 24 logits buffers
+    (184 MB at V = 32000, larger than L2), timed with CUDA events."""
+    import torch
+
+    B, H, T, D, V = cfg.B, cfg.H, cfg.T, cfg.D, cfg.V
+    i32 = dict(dtype=torch.int32, device=dev)
+    rng = np.random.default_rng(cfg.seed + 9)
+    NBUF = 24
+
+    def bench(fn, reps=30, inner=NBUF):
+        fn(0)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for j in range(inner):
+                fn(j)
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (reps * inner)
+
+    parents = np.stack([wl.eagle2_like_tree(rng, T, cfg.max_depth) for _ in range(B)]).astype(np.int32)
+    drafts = np.stack([wl.sibling_distinct_tokens(rng, p, V) for p in parents]).astype(np.int32)
+    par, drf = torch.tensor(parents, **i32), torch.tensor(drafts, **i32)
+    prefix_len = torch.tensor(wl.draw_prefix_lens(cfg, np.random.default_rng(cfg.seed)), **i32)
+    nb = max(2, min(NBUF, int(2.0e8 // (B * T * V * 4)) or 2))   # bounded memory for large batches
+    logits = [torch.randn((B, T, V), device=dev) for _ in range(nb)]
+    out = {}
+    # positioned inputs: rotate q and the tree's K rows, append K/V rows (one layer)
+    S_cap = cfg.s_cap
+    q = torch.randn((B, H, T, D), dtype=torch.bfloat16, device=dev)
+    kc = torch.zeros((B, H, S_cap, D), dtype=torch.bfloat16, device=dev)
+    vc = torch.zeros_like(kc)
+    qo = torch.empty_like(q)
+    out["rope_append_us"] = bench(lambda j: sv.specvlm_rope_append(q, q, q, prefix_len, par, qo, kc, vc))
+    # temperature > 0 acceptance (row statistics + walk + draw)
+    ua, us = torch.rand((B, T), device=dev), torch.rand((B, T), device=dev)
+    idx = torch.zeros((B, 8), **i32)
+    n, nx = torch.zeros(B, **i32), torch.zeros(B, **i32)
+    stats = torch.zeros((B, T, 2), device=dev)
+    out["accept_sample_us"] = bench(
+        lambda j: sv.specvlm_accept_sample(drf, par, logits[j % nb], ua, us, 1.0, idx, n, nx, stats))
+    # draft tree: top-10 log-probabilities of 10 expanded nodes per sequence, rerank of 511 candidates to T
+    k = 10
+    rows = [lg.view(B * T, V)[: 10 * B] for lg in logits]
+    tk, lp = torch.zeros((10 * B, k), **i32), torch.zeros((10 * B, k), device=dev)
+    out["topk_logprob_us"] = bench(lambda j: sv.specvlm_topk_logprob(rows[j % nb], k, tk, lp))
+    C = 511
+    cp = torch.zeros((B, C), **i32)
+    cp[:, 0] = -1
+    cs = -torch.rand((B, C), device=dev).cumsum(1)
+    ct = torch.zeros((B, C), **i32)
+    tp, dt = torch.zeros((B, T), **i32), torch.zeros((B, T), **i32)
+    out["tree_rerank_us"] = bench(lambda j: sv.specvlm_tree_rerank(cp, cs, ct, T, tp, dt))
+    # visual compression of one image's 2880 x 4096 features: 4x average pooling, pruning to a third
+    x = torch.randn((1, 2880, 4096), dtype=torch.bfloat16, device=dev)
+    y = torch.empty((1, 720, 4096), dtype=torch.bfloat16, device=dev)
+    out["visual_pool_us"] = bench(lambda j: sv.specvlm_visual_pool(x, 4, y))
+    keep = torch.arange(0, 2880, 3, **i32)[None].contiguous()
+    y2 = torch.empty((1, 960, 4096), dtype=torch.bfloat16, device=dev)
+    out["visual_prune_us"] = bench(lambda j: sv.specvlm_visual_prune(x, keep, y2))
+    out["note"] = ("microseconds per launch, CUDA-graph replay; logits rotate over "
+                   f"{nb} buffers of {B * T * V * 4 / 1e6:.1f} MB")
+    return {k_: (round(v, 2) if isinstance(v, float) else v) for k_, v in out.items()}
+
+
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -519,6 +595,8 @@ def run_ours(args, cfg):
             "gpu_launches": launches_per_step * args.steps, "launch_mode": "cuda_graph" if graphs_pipe else "python",
             "clocks": sampler.summary(),
         }
+        if world == 1:
+            line["widened_rows"] = time_widened_rows(sv, cfg, dev)
         if world == 1 and not args.no_cpu_baseline:
             piece, cores = oracle_sample(cfg, L)
             line["cpu_baseline"] = {
