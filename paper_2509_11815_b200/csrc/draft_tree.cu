@@ -210,37 +210,98 @@ topk_cluster_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
   }
   if (lane == 0) { s_m[warp] = m; s_z[warp] = z; }
 
-  // ---- k selection rounds inside every warp, no block-wide step: each round's winner is the best
-  // entry of the warp that comes strictly after the previous winner, found with two warp-wide
-  // integer reductions (largest order-preserving key, then lowest index among its holders);
-  // lane r keeps the winner of round r
-  Cand last{INFINITY, -1};
+  // ---- every warp finds the sorted top k of its own share, no block-wide step.
+  // Prefilter: the k-th best of the 32 lanes' own best entries (k rounds over one value per lane)
+  // is a threshold that at least k entries of the warp reach, so the warp's top k are among the
+  // entries that are not after it; typically fewer than 2 k entries pass. They are compacted into
+  // a short list with ballots and ranked by counting. If more than kListCap pass (a lane holding
+  // many of the warp's largest values), the warp falls back to k selection rounds over all of its
+  // registers.
+  constexpr int kListCap = 64;
+  __shared__ Cand s_list[kWarps][kListCap];
+  __shared__ Cand s_wl[kWarps * kMaxK];  // every warp's sorted top k
   Cand kept{-INFINITY, INT_MAX};
-  for (int r = 0; r < k; ++r) {
-    Cand c{-INFINITY, INT_MAX};
+  Cand lm{-INFINITY, INT_MAX};  // this lane's best entry: first maximum in (u, e) order = lowest index
 #pragma unroll
-    for (int u = 0; u < kU; ++u) {
+  for (int u = 0; u < kU; ++u) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int v = vbase + u * (kTkThreads * 4) + e;
-        const float val = vals[4 * u + e];
-        const bool after = val < last.v || (val == last.v && v > last.i);
-        if (after && val > c.v) c = Cand{val, v};  // first maximum in (u, e) order = lowest index
+    for (int e = 0; e < 4; ++e) {
+      const float val = vals[4 * u + e];
+      if (val > lm.v) lm = Cand{val, vbase + u * (kTkThreads * 4) + e};
+    }
+  }
+  Cand thr{-INFINITY, INT_MAX};
+  {
+    const unsigned lkey = ordered_key(lm.v);
+    bool used = false;
+    for (int r = 0; r < k; ++r) {
+      const unsigned key = used ? 0u : lkey;  // every real key is above 0
+      const unsigned kmax = __reduce_max_sync(0xffffffffu, key);
+      const unsigned imin =
+          __reduce_min_sync(0xffffffffu, (!used && key == kmax) ? static_cast<unsigned>(lm.i) : 0xffffffffu);
+      if (!used && key == kmax && static_cast<unsigned>(lm.i) == imin) used = true;
+      thr = Cand{key_value(kmax), static_cast<int>(imin)};
+    }
+    // lanes without any selectable entry report (-inf, INT_MAX): then every selectable entry passes
+    if (thr.i == INT_MAX || !(thr.v > -INFINITY)) thr = Cand{-INFINITY, INT_MAX};
+  }
+  int n_list = 0;  // warp-uniform
+#pragma unroll
+  for (int u = 0; u < kU; ++u) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int v = vbase + u * (kTkThreads * 4) + e;
+      const float val = vals[4 * u + e];
+      const bool pass = val > -INFINITY && (val > thr.v || (val == thr.v && v <= thr.i));
+      const unsigned ball = __ballot_sync(0xffffffffu, pass);
+      if (ball != 0u) {
+        const int slot = n_list + __popc(ball & ((1u << lane) - 1u));
+        if (pass && slot < kListCap) s_list[warp][slot] = Cand{val, v};
+        n_list += __popc(ball);
       }
     }
-    const unsigned key = ordered_key(c.v);
-    const unsigned kmax = __reduce_max_sync(0xffffffffu, key);
-    const unsigned imin = __reduce_min_sync(0xffffffffu, key == kmax ? static_cast<unsigned>(c.i) : 0xffffffffu);
-    // an exhausted warp reduces to (-inf, INT_MAX): INT_MAX is the smallest index any lane reports then
-    const Cand w{key_value(kmax), static_cast<int>(imin)};
-    last = w;
-    if (lane == r) kept = w;
   }
-  if (kept.i == INT_MAX) kept.i = kSentinel0 + (part * kWarps + warp) * kMaxK + lane;  // unique per entry
+  __syncwarp();
+  if (n_list <= kListCap) {
+    // rank by counting inside the list; places n_list .. k-1 (fewer than k selectable entries) stay empty
+    for (int q = lane; q < n_list; q += 32) {
+      const Cand me = s_list[warp][q];
+      int rank = 0;
+      for (int o = 0; o < n_list; ++o) rank += before(s_list[warp][o], me) ? 1 : 0;
+      if (rank < k) s_wl[warp * kMaxK + rank] = me;
+    }
+    // fewer than k selectable entries: the remaining places get sentinels, unique per entry
+    if (lane >= n_list && lane < k)
+      s_wl[warp * kMaxK + lane] = Cand{-INFINITY, kSentinel0 + (part * kWarps + warp) * kMaxK + lane};
+  } else {
+    // k selection rounds: each round's winner is the best entry that comes strictly after the
+    // previous winner, found with two warp-wide integer reductions; lane r keeps round r's winner
+    Cand last{INFINITY, -1};
+    for (int r = 0; r < k; ++r) {
+      Cand c{-INFINITY, INT_MAX};
+#pragma unroll
+      for (int u = 0; u < kU; ++u) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int v = vbase + u * (kTkThreads * 4) + e;
+          const float val = vals[4 * u + e];
+          const bool after = val < last.v || (val == last.v && v > last.i);
+          if (after && val > c.v) c = Cand{val, v};
+        }
+      }
+      const unsigned key = ordered_key(c.v);
+      const unsigned kmax = __reduce_max_sync(0xffffffffu, key);
+      const unsigned imin = __reduce_min_sync(0xffffffffu, key == kmax ? static_cast<unsigned>(c.i) : 0xffffffffu);
+      // an exhausted warp reduces to (-inf, INT_MAX): INT_MAX is the smallest index any lane reports then
+      const Cand w{key_value(kmax), static_cast<int>(imin)};
+      last = w;
+      if (lane == r) kept = w;
+    }
+    if (kept.i == INT_MAX) kept.i = kSentinel0 + (part * kWarps + warp) * kMaxK + lane;  // unique per entry
+    if (lane < k) s_wl[warp * kMaxK + lane] = kept;
+  }
   // ---- the warps' sorted lists are merged by counting
-  __shared__ Cand s_wl[kWarps * kMaxK];
   __shared__ Cand s_top[kMaxK];
-  if (lane < k) s_wl[warp * kMaxK + lane] = kept;
   __syncthreads();
   // Two threads per entry (entry = list * kMaxK + place), each searching half of the lists: with a
   // single warp per scheduler a chain of dependent instructions issues once every few cycles, so

@@ -25,6 +25,13 @@ def test_topk_logprob_matches_oracle(V, k, pad):
     if V >= 1000:
         x[3, 1::2] = -np.inf                                # masked vocabulary entries never win
         x[4, : V - 40] = -np.inf                            # everything finite sits in the last block's share
+    if V >= 8192:
+        # 16 lanes of one warp own all of the row's largest values (indices 4 t + e + 1024 u for the
+        # first block's thread t): too many entries pass the warp's prefilter, so its
+        # selection-round path runs
+        own = np.array([4 * t + e + 1024 * u for t in range(16) for u in range(4) for e in range(4)])
+        x[5, own] += 20.0
+        x[6, :64] = 30.0                                    # 64 equal maxima, ids decide
     store = torch.full((rows, V + pad), 1e30, dtype=torch.float32, device="cuda")   # padding must never win
     store[:, :V] = torch.from_numpy(x).cuda()
     lg = store[:, :V]
