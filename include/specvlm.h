@@ -363,6 +363,23 @@ SPECVLM_API int specvlm_verify_step(const uint16_t* q, int64_t q_stride_l, uint1
                         int32_t* next_token, int32_t* new_prefix_len, int layers_independent,
                         void* workspace, int32_t* status, void* stream);
 
+/*
+ * The verify step at temperature > 0 in one host call (Section 4.1 evaluates temperature 1; the
+ * target distribution is preserved): the L attention launches as in specvlm_verify_step, then
+ * specvlm_accept_sample (speculative sampling along the tree; row statistics, walk and draw), then
+ * specvlm_kv_compact over all layers. Arguments as in those calls; acc_stride must cover the
+ * deepest path (depth + 1 entries), since the compaction reads accepted_idx.
+ */
+SPECVLM_API int specvlm_verify_step_sample(const uint16_t* q, int64_t q_stride_l, uint16_t* k_cache,
+                        uint16_t* v_cache, const specvlm_kv_desc* kv_desc_host, const int32_t* prefix_len,
+                        const int32_t* tree_parent, const uint64_t* tree_mask_bits,
+                        const int32_t* draft_tokens, const float* target_logits,
+                        const float* uniforms_accept, const float* uniforms_sample, float temperature,
+                        int T, int V, uint16_t* out, int64_t out_stride_l, float* row_stats,
+                        int32_t* accepted_idx, int acc_stride, int32_t* accept_len, int32_t* next_token,
+                        int32_t* new_prefix_len, int layers_independent, void* workspace, int32_t* status,
+                        void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -40,6 +40,7 @@ EXPORTS = (
     "specvlm_kv_compact",
     "specvlm_accept_compact",
     "specvlm_verify_step",
+    "specvlm_verify_step_sample",
 )
 
 
@@ -129,6 +130,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.specvlm_accept_compact.restype = i32
     lib.specvlm_accept_compact.argtypes = [vp, vp, vp, i32, vp, vp, ctypes.POINTER(KvDesc), vp, vp, i32,
                                            vp, vp, vp, vp, vp]
+    lib.specvlm_verify_step_sample.restype = i32
+    lib.specvlm_verify_step_sample.argtypes = [vp, i64, vp, vp, ctypes.POINTER(KvDesc), vp, vp, vp, vp, vp, vp, vp,
+                                               ctypes.c_float, i32, i32, vp, i64, vp, vp, i32, vp, vp, vp, i32, vp, vp,
+                                               vp]
     lib.specvlm_verify_step.restype = i32
     lib.specvlm_verify_step.argtypes = [vp, i64, vp, vp, ctypes.POINTER(KvDesc), vp, vp, vp, vp, vp, i32, i32, vp, i64,
                                         vp, vp, i32, vp, vp, vp, i32, vp, vp, vp]
@@ -468,3 +473,36 @@ def specvlm_verify_step(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.T
         _ptr(tree_mask_bits), _ptr(draft_tokens), _ptr(target_logits), T, V, _ptr(out), out.stride(0),
         _ptr(argmax_tokens), _ptr(accepted_idx), accepted_idx.shape[1], _ptr(accept_len), _ptr(next_token),
         _ptr(new_prefix_len), 1 if layers_independent else 0, _ptr(workspace), _ptr(status), _stream()))
+
+
+def specvlm_verify_step_sample(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, prefix_len: torch.Tensor,
+                               tree_parent: torch.Tensor, tree_mask_bits: Optional[torch.Tensor],
+                               draft_tokens: torch.Tensor, target_logits: torch.Tensor, uniforms_accept: torch.Tensor,
+                               uniforms_sample: torch.Tensor, temperature: float, out: torch.Tensor,
+                               row_stats: torch.Tensor, accepted_idx: torch.Tensor, accept_len: torch.Tensor,
+                               next_token: torch.Tensor, new_prefix_len: torch.Tensor,
+                               layers_independent: bool = False, workspace: Optional[torch.Tensor] = None,
+                               status: Optional[torch.Tensor] = None) -> None:
+    """Whole verify step at temperature > 0 in one call; tensors as in specvlm_verify_step and
+    specvlm_accept_sample."""
+    desc = make_kv_desc(k_cache)
+    if tuple(v_cache.shape) != tuple(k_cache.shape) or v_cache.stride() != k_cache.stride():
+        raise SpecvlmError("k_cache and v_cache must share shape and strides")
+    _need(q, torch.bfloat16, "q")
+    _need(out, torch.bfloat16, "out")
+    if q.dim() != 5 or not q[0].is_contiguous() or not out[0].is_contiguous() or out.shape != q.shape:
+        raise SpecvlmError("q and out must be [L][B][H][T][D] with contiguous layers")
+    for name, t in (("target_logits", target_logits), ("uniforms_accept", uniforms_accept),
+                    ("uniforms_sample", uniforms_sample), ("row_stats", row_stats)):
+        _need(t, torch.float32, name)
+        if not t.is_contiguous():
+            raise SpecvlmError(f"{name} must be contiguous")
+    B, T, V = q.shape[1], q.shape[3], target_logits.shape[-1]
+    if row_stats.numel() != B * T * 2:
+        raise SpecvlmError("row_stats must hold B * T * 2 floats")
+    _check(load_library().specvlm_verify_step_sample(
+        _ptr(q), q.stride(0), _ptr(k_cache), _ptr(v_cache), ctypes.byref(desc), _ptr(prefix_len), _ptr(tree_parent),
+        _ptr(tree_mask_bits), _ptr(draft_tokens), _ptr(target_logits), _ptr(uniforms_accept), _ptr(uniforms_sample),
+        float(temperature), T, V, _ptr(out), out.stride(0), _ptr(row_stats), _ptr(accepted_idx),
+        accepted_idx.shape[1], _ptr(accept_len), _ptr(next_token), _ptr(new_prefix_len),
+        1 if layers_independent else 0, _ptr(workspace), _ptr(status), _stream()))

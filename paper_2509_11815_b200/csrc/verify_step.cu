@@ -2,17 +2,17 @@
 // launches (Sections 3.1, 3.2, 4.1), the vocabulary argmax, and the fused acceptance walk + KV
 // compaction (Section 3.1: incorrect tokens are discarded). It only chains the library's own
 // entry points on the caller's stream, so a caller without CUDA graphs pays one host call per
-// step instead of L + 2.
+// step instead of L + 2. specvlm_verify_step_sample is the temperature > 0 form: acceptance by
+// speculative sampling (Section 4.1 evaluates temperature 1), then the compaction.
 #include "common.cuh"
 
-extern "C" int specvlm_verify_step(const uint16_t* q, int64_t q_stride_l, uint16_t* k_cache, uint16_t* v_cache,
-                                   const specvlm_kv_desc* kv, const int32_t* prefix_len,
-                                   const int32_t* tree_parent, const uint64_t* tree_mask_bits,
-                                   const int32_t* draft_tokens, const float* target_logits, int T, int V,
-                                   uint16_t* out, int64_t out_stride_l, int32_t* argmax_tokens,
-                                   int32_t* accepted_idx, int acc_stride, int32_t* accept_len,
-                                   int32_t* next_token, int32_t* new_prefix_len, int layers_independent,
-                                   void* workspace, int32_t* status, void* stream) {
+namespace {
+
+// The L attention launches of a step; checks the arguments that both step entry points share.
+int attention_layers(const uint16_t* q, int64_t q_stride_l, uint16_t* k_cache, uint16_t* v_cache,
+                     const specvlm_kv_desc* kv, const int32_t* prefix_len, const int32_t* tree_parent,
+                     const uint64_t* tree_mask_bits, int T, uint16_t* out, int64_t out_stride_l,
+                     int layers_independent, void* workspace, int32_t* status, void* stream) {
   SPECVLM_REQUIRE(kv != nullptr, "verify_step: null kv descriptor");
   SPECVLM_REQUIRE(kv->L >= 1 && kv->D == SPECVLM_HEAD_DIM, "verify_step: need L >= 1 and D = 128");
   SPECVLM_REQUIRE(q && out && k_cache && v_cache, "verify_step: null pointer");
@@ -36,8 +36,43 @@ extern "C" int specvlm_verify_step(const uint16_t* q, int64_t q_stride_l, uint16
                                       workspace, status, stream);
     if (rc != SPECVLM_OK) return rc;
   }
-  int rc = specvlm_argmax(target_logits, kv->B, T, V, V, argmax_tokens, stream);
+  return SPECVLM_OK;
+}
+
+}  // namespace
+
+extern "C" int specvlm_verify_step(const uint16_t* q, int64_t q_stride_l, uint16_t* k_cache, uint16_t* v_cache,
+                                   const specvlm_kv_desc* kv, const int32_t* prefix_len,
+                                   const int32_t* tree_parent, const uint64_t* tree_mask_bits,
+                                   const int32_t* draft_tokens, const float* target_logits, int T, int V,
+                                   uint16_t* out, int64_t out_stride_l, int32_t* argmax_tokens,
+                                   int32_t* accepted_idx, int acc_stride, int32_t* accept_len,
+                                   int32_t* next_token, int32_t* new_prefix_len, int layers_independent,
+                                   void* workspace, int32_t* status, void* stream) {
+  int rc = attention_layers(q, q_stride_l, k_cache, v_cache, kv, prefix_len, tree_parent, tree_mask_bits, T, out,
+                            out_stride_l, layers_independent, workspace, status, stream);
+  if (rc != SPECVLM_OK) return rc;
+  rc = specvlm_argmax(target_logits, kv->B, T, V, V, argmax_tokens, stream);
   if (rc != SPECVLM_OK) return rc;
   return specvlm_accept_compact(draft_tokens, tree_parent, argmax_tokens, T, k_cache, v_cache, kv, prefix_len,
                                 accepted_idx, acc_stride, accept_len, next_token, new_prefix_len, status, stream);
+}
+
+extern "C" int specvlm_verify_step_sample(const uint16_t* q, int64_t q_stride_l, uint16_t* k_cache,
+                                          uint16_t* v_cache, const specvlm_kv_desc* kv, const int32_t* prefix_len,
+                                          const int32_t* tree_parent, const uint64_t* tree_mask_bits,
+                                          const int32_t* draft_tokens, const float* target_logits,
+                                          const float* uniforms_accept, const float* uniforms_sample,
+                                          float temperature, int T, int V, uint16_t* out, int64_t out_stride_l,
+                                          float* row_stats, int32_t* accepted_idx, int acc_stride,
+                                          int32_t* accept_len, int32_t* next_token, int32_t* new_prefix_len,
+                                          int layers_independent, void* workspace, int32_t* status, void* stream) {
+  int rc = attention_layers(q, q_stride_l, k_cache, v_cache, kv, prefix_len, tree_parent, tree_mask_bits, T, out,
+                            out_stride_l, layers_independent, workspace, status, stream);
+  if (rc != SPECVLM_OK) return rc;
+  rc = specvlm_accept_sample(draft_tokens, tree_parent, target_logits, uniforms_accept, uniforms_sample, temperature,
+                             kv->B, T, V, accepted_idx, acc_stride, accept_len, next_token, row_stats, status, stream);
+  if (rc != SPECVLM_OK) return rc;
+  return specvlm_kv_compact(k_cache, v_cache, kv, prefix_len, accepted_idx, acc_stride, accept_len, new_prefix_len,
+                            status, stream);
 }
