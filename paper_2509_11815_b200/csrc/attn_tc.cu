@@ -260,6 +260,9 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
 
   const bool inputs_stable = (p.flags & SPECVLM_ATTN_FLAG_INPUTS_STABLE) != 0;
   const bool prefix_stable = inputs_stable || (p.flags & SPECVLM_ATTN_FLAG_PREFIX_STABLE) != 0;
+  // With either promise prefix_len is not written by the preceding kernel: its load is issued
+  // first, so that its latency runs beside the set-up below instead of after it.
+  int prefix_raw = prefix_stable ? p.prefix_len[b] : 0;
 
   // ---- set-up that touches no global input: tensor-map prefetch, barriers, TMEM
   if (threadIdx.x == 0) {
@@ -282,9 +285,11 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
   // Without a promise from the caller, nothing below may run before the preceding kernel has
   // completed. Only then is the next launch allowed to start: a successor that was promised stable
   // inputs must not overtake work that this kernel itself still had to wait for.
-  if (!prefix_stable) pdl_wait();
+  if (!prefix_stable) {
+    pdl_wait();
+    prefix_raw = p.prefix_len[b];
+  }
   pdl_launch_dependents();
-  const int prefix_raw = p.prefix_len[b];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
