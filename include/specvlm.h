@@ -76,7 +76,11 @@ extern "C" {
  * INPUTS_STABLE: nothing this call reads (q, caches, prefix_len, tree arrays) is written by the
  *   preceding kernel: the whole call may overlap with it (back-to-back attention calls on
  *   independent inputs, as in a benchmark). Its writes to `out` are still issued only after the
- *   preceding kernel has completed. */
+ *   preceding kernel has completed. A launch with this flag lets its own successor start at
+ *   once, so in a run of consecutive INPUTS_STABLE launches each may overlap all launches of the
+ *   run before it and the kernel before the run: the promise must hold against all of those.
+ * A launch without INPUTS_STABLE lets its successor start only after its own wait for the
+ * preceding kernel is over, so everything earlier on the stream is complete by then. */
 #define SPECVLM_ATTN_FLAG_PREFIX_STABLE 2
 #define SPECVLM_ATTN_FLAG_INPUTS_STABLE 4
 /* Run in the configuration that occupies half an SM per thread block (chosen automatically for

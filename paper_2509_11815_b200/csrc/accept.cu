@@ -24,6 +24,7 @@ __global__ void tree_build_kernel(const int32_t* __restrict__ parent, const int3
   const int i = threadIdx.x;
   __shared__ int s_parent[kMaxT];
   __shared__ int s_bad;
+  grid_dependency_sync();
   if (i == 0) s_bad = 0;
   __syncthreads();
   if (i < T) {
@@ -214,6 +215,7 @@ accept_compact_kernel(const int32_t* __restrict__ draft, const int32_t* __restri
                       int32_t* __restrict__ new_prefix_len, int32_t* __restrict__ status) {
   __shared__ int s_parent[kMaxT], s_ok[kMaxT], s_path[kMaxT], s_scratch[2];
   const int b = blockIdx.y;
+  grid_dependency_sync();
   const int P = prefix_len[b];
   WalkResult r = walk_tree(draft + b * T, parent + b * T, tok + b * T, T, s_parent, s_ok, s_path,
                            s_scratch, blockIdx.x == 0 ? status : nullptr);
@@ -269,9 +271,9 @@ extern "C" int specvlm_tree_build(const int32_t* tree_parent, const int32_t* pre
   if (B == 0) return SPECVLM_OK;
   SPECVLM_REQUIRE(tree_parent != nullptr && mask_bits != nullptr, "tree_build: null pointer");
   SPECVLM_REQUIRE(pos == nullptr || prefix_len != nullptr, "tree_build: pos needs prefix_len");
-  tree_build_kernel<<<B, kMaxT, 0, static_cast<cudaStream_t>(stream)>>>(tree_parent, prefix_len, B, T,
-                                                                       mask_bits, depth, pos, status);
-  return check_cuda(cudaGetLastError(), "tree_build launch");
+  return check_cuda(launch_overlapped(tree_build_kernel, dim3(B), dim3(kMaxT), static_cast<cudaStream_t>(stream),
+                                      tree_parent, prefix_len, B, T, mask_bits, depth, pos, status),
+                    "tree_build launch");
 }
 
 extern "C" int specvlm_accept(const int32_t* draft_tokens, const int32_t* tree_parent,
@@ -328,8 +330,9 @@ extern "C" int specvlm_accept_compact(const int32_t* draft_tokens, const int32_t
   SPECVLM_REQUIRE(new_prefix_len != prefix_len, "accept_compact: new_prefix_len must not alias prefix_len");
   SPECVLM_REQUIRE(acc_stride >= 1, "accept_compact: acc_stride must be >= 1");
   dim3 grid(compact_grid_x(desc), desc->B);
-  accept_compact_kernel<<<grid, kCompactThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      draft_tokens, tree_parent, argmax_tokens, T, make_kv_params(k_cache, v_cache, desc), prefix_len,
-      accepted_idx, acc_stride, accept_len, next_token, new_prefix_len, status);
-  return check_cuda(cudaGetLastError(), "accept_compact launch");
+  return check_cuda(launch_overlapped(accept_compact_kernel, grid, dim3(kCompactThreads),
+                                      static_cast<cudaStream_t>(stream), draft_tokens, tree_parent, argmax_tokens, T,
+                                      make_kv_params(k_cache, v_cache, desc), prefix_len, accepted_idx, acc_stride,
+                                      accept_len, next_token, new_prefix_len, status),
+                    "accept_compact launch");
 }

@@ -48,6 +48,7 @@ argmax_rows_kernel(const float* __restrict__ logits, int V, int64_t row_stride,
   const int per = (n4 + kArgmaxSplit - 1) / kArgmaxSplit;
   const int g0 = part * per, g1 = min(g0 + per, n4);
 
+  grid_dependency_sync();
   cluster.barrier_arrive();  // matched by the wait below: every CTA of the cluster has started by then
   Best best{-INFINITY, INT_MAX};
   // -inf never passes '>' against the initial -inf; INT_MAX then loses every index tie,
@@ -107,13 +108,15 @@ int launch_argmax(const float* logits, int rows, int V, int64_t row_stride, int3
   cfg.blockDim = dim3(kArgmaxThreads);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = kArgmaxSplit;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the kernel starts with grid_dependency_sync()
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return check_cuda(cudaLaunchKernelEx(&cfg, argmax_rows_kernel, logits, V, row_stride, out), "argmax launch");
 }
 

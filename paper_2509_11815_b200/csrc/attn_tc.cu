@@ -288,8 +288,11 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
   if (!prefix_stable) {
     pdl_wait();
     prefix_raw = p.prefix_len[b];
+    pdl_launch_dependents();
+  } else if (inputs_stable) {
+    pdl_launch_dependents();  // this launch never waits before it reads
   }
-  pdl_launch_dependents();
+  // PREFIX_STABLE alone: the producer lets the next launch start once its own wait is over
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -350,6 +353,7 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
         while (ik < n_tiles && ik < kKStages && KEY0(ik) + kTile <= P) issue_k(ik++);
         while (iv < n_tiles && iv < kVStages && KEY0(iv) + kTile <= P) issue_v(iv++);
         pdl_wait();
+        pdl_launch_dependents();
       }
       issue_q();
       uint32_t idle = 0;
