@@ -65,6 +65,7 @@ softmax_stats_kernel(const float* __restrict__ logits, int V, float inv_temp, in
   cg::cluster_group cluster = cg::this_cluster();
   const int row = blockIdx.x / kStatSplit, part = blockIdx.x % kStatSplit;  // part == rank in the cluster
   const float* x = logits + static_cast<int64_t>(row) * V;
+  grid_dependency_sync();
   cluster.barrier_arrive();  // matched by the wait before the first remote store
   Stat st{-INFINITY, 0.f};
   if (vec) {
@@ -170,13 +171,19 @@ accept_sample_kernel(const int32_t* __restrict__ draft, const int32_t* __restric
         if (s_draft[c] == x) usable = false;
       }
     }
+    s_usable[t] = usable ? 1 : 0;
+  }
+  // Everything above reads only this call's inputs, which no kernel that may still be running
+  // writes; the row statistics come from the launch just before this one.
+  const float child_logit = (t < T && s_usable[t]) ? logits[static_cast<int64_t>(pr) * V + x] : 0.f;
+  grid_dependency_sync();
+  if (t < T) {
     float px = 0.f;
-    if (usable) {
+    if (s_usable[t]) {
       const float2 mz = stats[pr];
-      px = __expf((logits[static_cast<int64_t>(pr) * V + x] - mz.x) * inv_temp) / mz.y;
+      px = __expf((child_logit - mz.x) * inv_temp) / mz.y;
     }
     s_px[t] = px;
-    s_usable[t] = usable ? 1 : 0;
   }
   __syncthreads();
 
@@ -368,19 +375,24 @@ extern "C" int specvlm_accept_sample(const int32_t* draft_tokens, const int32_t*
     cfg.gridDim = dim3(static_cast<unsigned>(kStatSplit) * B * T);  // rows along x: no 65535 limit
     cfg.blockDim = dim3(kStatThreads);
     cfg.stream = static_cast<cudaStream_t>(stream);
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = kStatSplit;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the kernel starts with grid_dependency_sync()
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     const int rc = check_cuda(cudaLaunchKernelEx(&cfg, softmax_stats_kernel, target_logits, V, inv_temp, vec, stats),
                               "accept_sample row statistics launch");
     if (rc != SPECVLM_OK) return rc;
   }
-  accept_sample_kernel<<<B, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      draft_tokens, tree_parent, target_logits, stats, uniforms_accept, uniforms_sample, inv_temp, T, V,
-      accepted_idx, acc_stride, accept_len, next_token, status);
-  return check_cuda(cudaGetLastError(), "accept_sample launch");
+  // The walk kernel is scheduled while the statistics kernel runs: it reads its own inputs, then
+  // waits for the statistics.
+  return check_cuda(launch_overlapped(accept_sample_kernel, dim3(B), dim3(kSampleThreads),
+                                      static_cast<cudaStream_t>(stream), draft_tokens, tree_parent, target_logits,
+                                      static_cast<const float2*>(stats), uniforms_accept, uniforms_sample, inv_temp,
+                                      T, V, accepted_idx, acc_stride, accept_len, next_token, status),
+                    "accept_sample launch");
 }

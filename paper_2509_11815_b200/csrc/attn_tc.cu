@@ -208,13 +208,6 @@ __device__ __forceinline__ void st_cluster_f32x2(uint32_t addr, float a, float b
   asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
 
-#ifdef SPECVLM_TC_TRACE
-__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define TRACE(slot) do { if (trace_on) trace[(slot)] = gtime(); } while (0)
-#else
-#define TRACE(slot) do { } while (0)
-#endif
-
 }  // namespace tc
 
 using namespace tc;
@@ -239,11 +232,6 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int T = p.T;
-#ifdef SPECVLM_TC_TRACE
-  long long* trace = reinterpret_cast<long long*>(p.counters) + 64 * (blockIdx.y * gridDim.x + blockIdx.x);
-  const bool trace_on = p.counters != nullptr && lane == 0 && blockIdx.z == 0;
-  if (warp <= 2) TRACE(warp);
-#endif
 
   // barrier addresses: full_k[] empty_k[] full_v[] empty_v[] s_full[2] s_free[2] p_full pv_done q_full land_full
   const uint32_t bar0 = base + kOffBar;
@@ -297,9 +285,6 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-#ifdef SPECVLM_TC_TRACE
-  if (warp <= 2) TRACE(3 + warp);
-#endif
 
   // ---- sequence geometry
   int P = prefix_raw;
@@ -344,7 +329,6 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
         const uint32_t dv = base + kOffV + sv * kVBytes;
         mbar_expect_tx(FULL_V(sv), kVBytes);
         tma_load_rows(dv, &map_v, FULL_V(sv), KEY0(i), h, b);
-        TRACE(8 + (i < 12 ? i : 12));
       };
       int ik = 0, iv = 0;
       if (prefix_stable && !inputs_stable) {
@@ -425,18 +409,12 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
         bool progress = false;
         if (ip < iq && mbar_try_wait(P_FULL, ip & 1) && mbar_try_wait(FULL_V(ip % kVStages), (ip / kVStages) & 1)) {
           tc_fence_after();
-#ifdef SPECVLM_TC_TRACE
-          if (ip < 8) TRACE(47 + 2 * ip);
-#endif
           issue_pv(ip++);
           progress = true;
         }
         if (iq < n_tiles && iq < ip + 2 && mbar_try_wait(FULL_K(iq % kKStages), (iq / kKStages) & 1) &&
             (iq < 2 || mbar_try_wait(S_FREE(iq & 1), ((iq >> 1) & 1) ^ 1))) {
           tc_fence_after();
-#ifdef SPECVLM_TC_TRACE
-          if (iq < 8) TRACE(48 + 2 * iq);
-#endif
           issue_qk(iq++);
           progress = true;
         }
@@ -600,9 +578,6 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
       tc_fence_before();
       mbar_arrive(P_FULL);
-#ifdef SPECVLM_TC_TRACE
-      if (warp == 2) TRACE(24 + (i < 12 ? i : 12));
-#endif
     }
     if (ok && n_tiles > 0) {
       ok = mbar_wait(PV_DONE, (n_tiles - 1) & 1, abort_flag);
@@ -613,9 +588,6 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
   }
-#ifdef SPECVLM_TC_TRACE
-  if (warp <= 2) TRACE(40 + warp);
-#endif
 
   uint16_t* obase = p.out + b * p.o_sb + h * p.o_sh;
   const bool have_o = n_tiles > 0;  // otherwise the TMEM accumulator was never written
@@ -698,15 +670,9 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // staging is read by the bulk copies
   }
-#ifdef SPECVLM_TC_TRACE
-  if (warp == 2) TRACE(43);
-#endif
   tc_fence_before();
   cluster.sync();
   tc_fence_after();
-#ifdef SPECVLM_TC_TRACE
-  if (warp == 2) TRACE(44);
-#endif
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
@@ -722,9 +688,6 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
   bool landed = true;
   if (warp >= kSoftmaxWarp0) landed = mbar_wait(LAND_FULL, 0, abort_flag);
   cluster.barrier_arrive();
-#ifdef SPECVLM_TC_TRACE
-  if (warp == 2) TRACE(45);
-#endif
   const bool aborted = *abort_flag != 0;
   if (aborted && threadIdx.x == 0 && p.status != nullptr) atomicOr(p.status, SPECVLM_STATUS_TIMEOUT);
   if (warp >= kSoftmaxWarp0 && !aborted && landed) {
@@ -769,9 +732,6 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
       }
     }
   }
-#ifdef SPECVLM_TC_TRACE
-  if (warp == 2) TRACE(46);
-#endif
   cluster.barrier_wait();
 }
 
