@@ -338,3 +338,30 @@ def test_randomized_shape_sweep():
         got, status = run_attn(q, k, v, pl, masks=masks, num_splits=splits)
         assert status == 0, (trial, B, H, T, prefixes, splits)
         assert_attn_close(got, ref)
+
+
+@pytest.mark.parametrize("B,H,T", [(50, 8, 26), (23, 40, 60)])
+def test_more_items_than_resident_blocks(B, H, T):
+    """B * H above two blocks per SM, so the launch runs in more than one wave of blocks. Ragged
+    prefixes, including empty ones and a sequence whose prefix does not fit the cache (reported,
+    rows written as zeros)."""
+    rng = np.random.default_rng(B * H)
+    prefixes = rng.integers(0, 300, size=B)
+    prefixes[3] = 0
+    prefixes[B - 1] = 0
+    prefixes[B // 2] = 299
+    q, k, v, pl, parents, masks = make_case(4242 + B, B=B, H=H, T=T, prefixes=prefixes.tolist(), slack=3)
+    ref = oracle_attn_all(q, k, v, pl, masks)
+    got, status = run_attn(q, k, v, pl, masks=masks, num_splits=1)
+    assert status == 0
+    assert_attn_close(got, ref)
+    got2, status = run_attn(q, k, v, pl, parents=parents, num_splits=1)   # masks derived in the kernel
+    assert status == 0 and np.array_equal(got, got2)
+    # one sequence in the middle with an impossible prefix: flagged, its rows are zeros, the rest unchanged
+    bad = pl.copy()
+    bad[5] = 10_000
+    got3, status = run_attn(q, k, v, bad, masks=masks, num_splits=1, out_fill=7.0)
+    assert status & sv.STATUS_BAD_PREFIX
+    assert not got3[5].any()
+    keep = np.arange(B) != 5
+    assert np.array_equal(got3[keep], got[keep])
