@@ -125,6 +125,7 @@ accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ par
               int32_t* __restrict__ status) {
   __shared__ int s_parent[kMaxT], s_ok[kMaxT], s_path[kMaxT], s_scratch[2];
   const int b = blockIdx.x;
+  grid_dependency_sync();
   WalkResult r = walk_tree(draft + b * T, parent + b * T, tok + b * T, T, s_parent, s_ok, s_path,
                            s_scratch, status);
   write_accept_outputs(r, s_path, tok + b * T, b, accepted_idx, acc_stride, accept_len, next_token);
@@ -189,6 +190,7 @@ kv_compact_kernel(KvParams p, const int32_t* __restrict__ prefix_len, const int3
   __shared__ int s_path[kMaxT];
   __shared__ int s_good;
   const int b = blockIdx.y;
+  grid_dependency_sync();
   const int P = prefix_len[b];
   const int n = accept_len[b];
   if (threadIdx.x < kMaxT)
@@ -292,9 +294,10 @@ extern "C" int specvlm_accept(const int32_t* draft_tokens, const int32_t* tree_p
     int rc = launch_argmax(target_logits, B * T, V, V, argmax_tokens, s);
     if (rc != SPECVLM_OK) return rc;
   }
-  accept_kernel<<<B, kMaxT, 0, s>>>(draft_tokens, tree_parent, argmax_tokens, T, accepted_idx, acc_stride,
-                                    accept_len, next_token, status);
-  return check_cuda(cudaGetLastError(), "accept launch");
+  return check_cuda(launch_overlapped(accept_kernel, dim3(B), dim3(kMaxT), s, draft_tokens, tree_parent,
+                                      static_cast<const int32_t*>(argmax_tokens), T, accepted_idx, acc_stride,
+                                      accept_len, next_token, status),
+                    "accept launch");
 }
 
 extern "C" int specvlm_kv_compact(uint16_t* k_cache, uint16_t* v_cache, const specvlm_kv_desc* desc,
@@ -308,10 +311,10 @@ extern "C" int specvlm_kv_compact(uint16_t* k_cache, uint16_t* v_cache, const sp
   SPECVLM_REQUIRE(new_prefix_len != prefix_len, "kv_compact: new_prefix_len must not alias prefix_len");
   SPECVLM_REQUIRE(acc_stride >= 1, "kv_compact: acc_stride must be >= 1");
   dim3 grid(compact_grid_x(desc), desc->B);
-  kv_compact_kernel<<<grid, kCompactThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      make_kv_params(k_cache, v_cache, desc), prefix_len, accepted_idx, acc_stride, accept_len,
-      new_prefix_len, status);
-  return check_cuda(cudaGetLastError(), "kv_compact launch");
+  return check_cuda(launch_overlapped(kv_compact_kernel, grid, dim3(kCompactThreads), static_cast<cudaStream_t>(stream),
+                                      make_kv_params(k_cache, v_cache, desc), prefix_len, accepted_idx, acc_stride,
+                                      accept_len, new_prefix_len, status),
+                    "kv_compact launch");
 }
 
 extern "C" int specvlm_accept_compact(const int32_t* draft_tokens, const int32_t* tree_parent,

@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(kRopeThreads) rope_append_kernel(const RopePar
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   __shared__ float s_cos[64], s_sin[64];
   __shared__ int s_pos;
+  grid_dependency_sync();
   if (threadIdx.x == 0) {
     // depth by walking the parent chain (bounded even for a malformed tree)
     const int32_t* par = p.parent + b * p.T;
@@ -145,6 +146,6 @@ extern "C" int specvlm_rope_append(const uint16_t* q_in, const uint16_t* k_new, 
   int gz = (d->H + 2 * (kRopeThreads / 32) - 1) / (2 * (kRopeThreads / 32));
   if (static_cast<int64_t>(gz) * d->T * d->B > 4096) gz = 1;
   dim3 grid(d->T, d->B, gz);
-  rope_append_kernel<<<grid, kRopeThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
-  return check_cuda(cudaGetLastError(), "rope_append launch");
+  return check_cuda(launch_overlapped(rope_append_kernel, grid, dim3(kRopeThreads), static_cast<cudaStream_t>(stream), p),
+                    "rope_append launch");
 }
