@@ -375,30 +375,42 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
     if (lane == 0 && n_tiles > 0) {
       constexpr uint32_t idesc_qk = make_idesc(kTile, false), idesc_pv = make_idesc(kD, true);
       const uint32_t tmem_o = tmem_base + kColO;
+      // This one thread issues every MMA, and a lone thread issues a dependent instruction only
+      // every few cycles, so the per-MMA instruction count matters. Matrix descriptors of one
+      // operand buffer differ only in their start-address field (byte address >> 4, 14 bits, and
+      // shared-memory addresses stay below 2^18): one descriptor per buffer is built up front and
+      // moving it is one addition. Ring stages and barrier parities are carried along instead of
+      // being recomputed with divisions.
+      const uint64_t q_desc = make_desc(base + kOffQ, 16, 1024);
+      const uint64_t p_desc = make_desc(base + kOffP, 16, 1024);
+      const uint64_t k_desc0 = make_desc(base + kOffK, 16, 1024);
+      const uint64_t v_desc0 = make_desc(base + kOffV, kVBytes / 2, 1024);
+      int k_stage = 0, v_stage = 0;         // ring stage of the next S = Q K^T / the next O += P V
+      uint32_t k_parity = 0, v_parity = 0;  // parity of that stage's "full" barrier
       auto issue_qk = [&](int i) {
-        const int sk = i % kKStages;
-        const uint32_t ak = base + kOffK + sk * kKBytes;
+        const uint64_t kd = k_desc0 + static_cast<uint64_t>(k_stage * (kKBytes >> 4));
         const uint32_t tmem_s = tmem_base + ((i & 1) ? kColS1 : kColS0);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-          const uint64_t ad = make_desc(base + kOffQ + (ks >> 2) * (kQBytes / 2) + (ks & 3) * 32, 16, 1024);
-          const uint64_t bd = make_desc(ak + (ks >> 2) * (kKBytes / 2) + (ks & 3) * 32, 16, 1024);
+          const uint64_t ad = q_desc + static_cast<uint64_t>(((ks >> 2) * (kQBytes / 2) + (ks & 3) * 32) >> 4);
+          const uint64_t bd = kd + static_cast<uint64_t>(((ks >> 2) * (kKBytes / 2) + (ks & 3) * 32) >> 4);
           tc_mma(tmem_s, ad, bd, idesc_qk, ks > 0 ? 1u : 0u);
         }
-        tc_commit(EMPTY_K(sk));  // K stage free once these MMAs have read it
+        tc_commit(EMPTY_K(k_stage));  // K stage free once these MMAs have read it
         tc_commit(S_FULL(i & 1));
+        if (++k_stage == kKStages) { k_stage = 0; k_parity ^= 1u; }
       };
       auto issue_pv = [&](int i) {
-        const int sv = i % kVStages;
-        const uint32_t av = base + kOffV + sv * kVBytes;
+        const uint64_t vd = v_desc0 + static_cast<uint64_t>(v_stage * (kVBytes >> 4));
 #pragma unroll
         for (int ks = 0; ks < kTile / 16; ++ks) {
-          const uint64_t ad = make_desc(base + kOffP + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
-          const uint64_t bd = make_desc(av + ks * 2048, kVBytes / 2, 1024);
+          const uint64_t ad = p_desc + static_cast<uint64_t>(((ks >> 2) * 8192 + (ks & 3) * 32) >> 4);
+          const uint64_t bd = vd + static_cast<uint64_t>((ks * 2048) >> 4);
           tc_mma(tmem_o, ad, bd, idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
         }
-        tc_commit(EMPTY_V(sv));
+        tc_commit(EMPTY_V(v_stage));
         tc_commit(PV_DONE);
+        if (++v_stage == kVStages) { v_stage = 0; v_parity ^= 1u; }
       };
       // Whichever of "O += P V of tile ip" and "S = Q K^T of tile iq" has its operands ready is
       // issued; PV is looked at first because the softmax warps wait for its completion.
@@ -407,12 +419,12 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
       uint32_t idle = 0;
       while (ok && ip < n_tiles) {
         bool progress = false;
-        if (ip < iq && mbar_try_wait(P_FULL, ip & 1) && mbar_try_wait(FULL_V(ip % kVStages), (ip / kVStages) & 1)) {
+        if (ip < iq && mbar_try_wait(P_FULL, ip & 1) && mbar_try_wait(FULL_V(v_stage), v_parity)) {
           tc_fence_after();
           issue_pv(ip++);
           progress = true;
         }
-        if (iq < n_tiles && iq < ip + 2 && mbar_try_wait(FULL_K(iq % kKStages), (iq / kKStages) & 1) &&
+        if (iq < n_tiles && iq < ip + 2 && mbar_try_wait(FULL_K(k_stage), k_parity) &&
             (iq < 2 || mbar_try_wait(S_FREE(iq & 1), ((iq >> 1) & 1) ^ 1))) {
           tc_fence_after();
           issue_qk(iq++);
