@@ -365,3 +365,39 @@ def test_more_items_than_resident_blocks(B, H, T):
     assert not got3[5].any()
     keep = np.arange(B) != 5
     assert np.array_equal(got3[keep], got[keep])
+
+
+def test_invariance_under_prefix_permutation_and_tree_relabelling():
+    """Properties that hold at any size: jointly permuting the prefix rows of K and V changes only
+    the summation order; relabelling the tree nodes in another parent-before-child order permutes
+    slots, mask bits and output rows together."""
+    rng = np.random.default_rng(99)
+    B, H, T, P = 1, 4, 40, 777
+    q, k, v, pl, parents, masks = make_case(99, B=B, H=H, T=T, prefixes=[P])
+    base, status = run_attn(q, k, v, pl, masks=masks)
+    assert status == 0
+    perm = rng.permutation(P)
+    k2, v2 = k.copy(), v.copy()
+    k2[:, :, :P] = k[:, :, perm]
+    v2[:, :, :P] = v[:, :, perm]
+    got, status = run_attn(q, k2, v2, pl, masks=masks)
+    assert status == 0
+    d = np.abs(oracle.bf16_bits_to_f64(got) - oracle.bf16_bits_to_f64(base))
+    assert d.max() <= 2e-3, d.max()
+    # relabel: a random order in which every parent still precedes its children
+    parent = parents[0]
+    depth = oracle.tree_depth(parent)
+    order = np.lexsort((rng.random(T), depth))          # new label j <- old node order[j]
+    assert order[0] == 0
+    new_of_old = np.empty(T, dtype=np.int64)
+    new_of_old[order] = np.arange(T)
+    parent2 = np.array([-1] + [new_of_old[parent[order[j]]] for j in range(1, T)], dtype=np.int32)
+    assert oracle.is_valid_tree(parent2)
+    q3, k3, v3 = q.copy(), k.copy(), v.copy()
+    q3[:, :, :] = q[:, :, order]
+    k3[:, :, P:P + T] = k[:, :, P + order]
+    v3[:, :, P:P + T] = v[:, :, P + order]
+    got3, status = run_attn(q3, k3, v3, pl, masks=[oracle.tree_mask_bits(parent2)])
+    assert status == 0
+    d = np.abs(oracle.bf16_bits_to_f64(got3) - oracle.bf16_bits_to_f64(base[:, :, order]))
+    assert d.max() <= 2e-3, d.max()
