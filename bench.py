@@ -225,7 +225,7 @@ def workload_config(cfg):
 # ----------------------------------------------------------------------------- GPU arm
 
 
-def time_widened_rows(sv, cfg, dev):
+def time_widened_rows(sv, cfg, dev, k_cache, v_cache):
     """Microseconds per launch of the kernels next to the verify step (positioned inputs, temperature > 0
     acceptance, draft-tree construction, parameter-free visual compression) at this workload's shapes.
     Each kernel is replayed from a CUDA graph of 24 launches that rotate over 24 logits buffers
@@ -261,13 +261,18 @@ def time_widened_rows(sv, cfg, dev):
     nb = max(2, min(NBUF, int(2.0e8 // (B * T * V * 4)) or 2))   # bounded memory for large batches
     logits = [torch.randn((B, T, V), device=dev) for _ in range(nb)]
     out = {}
-    # positioned inputs: rotate q and the tree's K rows, append K/V rows (one layer)
-    S_cap = cfg.s_cap
-    q = torch.randn((B, H, T, D), dtype=torch.bfloat16, device=dev)
-    kc = torch.zeros((B, H, S_cap, D), dtype=torch.bfloat16, device=dev)
-    vc = torch.zeros_like(kc)
-    qo = torch.empty_like(q)
-    out["rope_append_us"] = bench(lambda j: sv.specvlm_rope_append(q, q, q, prefix_len, par, qo, kc, vc))
+    # positioned inputs: rotate q and the tree's K rows, append K/V rows, one launch per layer into
+    # the workload's own L caches (the appended rows of a layer's heads lie in different pages)
+    L = k_cache.shape[0]
+    qi, kn, vn = (torch.randn((L, B, H, T, D), dtype=torch.bfloat16, device=dev) for _ in range(3))
+    qo = torch.empty_like(qi)
+
+    def rope(j):
+        l = j % L
+        sv.specvlm_rope_append(qi[l], kn[l], vn[l], prefix_len, par, qo[l], k_cache[l], v_cache[l])
+
+    out["rope_append_us"] = bench(rope, inner=L)
+    del qi, kn, vn, qo
     # temperature > 0 acceptance (row statistics + walk + draw)
     ua, us = torch.rand((B, T), device=dev), torch.rand((B, T), device=dev)
     idx = torch.zeros((B, 8), **i32)
@@ -596,7 +601,7 @@ def run_ours(args, cfg):
             "clocks": sampler.summary(),
         }
         if world == 1:
-            line["widened_rows"] = time_widened_rows(sv, cfg, dev)
+            line["widened_rows"] = time_widened_rows(sv, cfg, dev, k_cache, v_cache)
         if world == 1 and not args.no_cpu_baseline:
             piece, cores = oracle_sample(cfg, L)
             line["cpu_baseline"] = {

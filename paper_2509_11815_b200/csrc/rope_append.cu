@@ -45,6 +45,7 @@ __global__ void __launch_bounds__(kRopeThreads) rope_append_kernel(const RopePar
   __shared__ float s_cos[64], s_sin[64];
   __shared__ int s_pos;
   grid_dependency_sync();
+  const int prefix = p.prefix_len[b];  // every thread: its latency runs beside the parent walk
   if (threadIdx.x == 0) {
     // depth by walking the parent chain (bounded even for a malformed tree)
     const int32_t* par = p.parent + b * p.T;
@@ -57,7 +58,7 @@ __global__ void __launch_bounds__(kRopeThreads) rope_append_kernel(const RopePar
       ++depth;
     }
     if (t == 0 && par[0] != -1) bad = true;
-    const int P = p.prefix_len[b];
+    const int P = prefix;
     const bool bad_prefix = P < 0 || P + p.T > p.S_cap;
     if (p.status != nullptr) {
       if (bad) atomicOr(p.status, SPECVLM_STATUS_BAD_TREE);
@@ -81,28 +82,31 @@ __global__ void __launch_bounds__(kRopeThreads) rope_append_kernel(const RopePar
   __syncthreads();
   // lane owns pairs d = 2*lane, 2*lane + 1 (elements d and d + 64)
   const float c0 = s_cos[2 * lane], s0 = s_sin[2 * lane], c1 = s_cos[2 * lane + 1], s1 = s_sin[2 * lane + 1];
-  const int slot = p.prefix_len[b] + t;
+  const int slot = prefix + t;
   for (int h = blockIdx.z * (kRopeThreads / 32) + warp; h < p.H; h += gridDim.z * (kRopeThreads / 32)) {
+    // all six loads of a head's rows are issued before its first store: q_out may alias q_in,
+    // which the compiler has to assume and would otherwise serialise three memory round trips
+    const uint32_t* qs = reinterpret_cast<const uint32_t*>(p.q_in + b * p.qi_sb + h * p.qi_sh + t * p.qi_st);
+    const uint32_t* ks = reinterpret_cast<const uint32_t*>(p.k_new + b * p.kn_sb + h * p.kn_sh + t * p.kn_st);
+    const uint32_t* vs = reinterpret_cast<const uint32_t*>(p.v_new + b * p.vn_sb + h * p.vn_sh + t * p.vn_st);
+    const uint32_t q_lo = qs[lane], q_hi = qs[lane + 32];
+    const uint32_t k_lo = ks[lane], k_hi = ks[lane + 32];
+    const uint32_t v_lo = vs[lane], v_hi = vs[lane + 32];
+    uint32_t* qd = reinterpret_cast<uint32_t*>(p.q_out + b * p.qo_sb + h * p.qo_sh + t * p.qo_st);
+    uint32_t* kd = reinterpret_cast<uint32_t*>(p.k_cache + b * p.kc_sb + h * p.kc_sh + slot * p.kc_ss);
+    uint32_t* vd = reinterpret_cast<uint32_t*>(p.v_cache + b * p.vc_sb + h * p.vc_sh + slot * p.vc_ss);
     {
-      const uint32_t* src = reinterpret_cast<const uint32_t*>(p.q_in + b * p.qi_sb + h * p.qi_sh + t * p.qi_st);
-      uint32_t* dst = reinterpret_cast<uint32_t*>(p.q_out + b * p.qo_sb + h * p.qo_sh + t * p.qo_st);
-      const float2 lo = unpack2(src[lane]), hi = unpack2(src[lane + 32]);
-      dst[lane] = pack2(lo.x * c0 - hi.x * s0, lo.y * c1 - hi.y * s1);
-      dst[lane + 32] = pack2(hi.x * c0 + lo.x * s0, hi.y * c1 + lo.y * s1);
+      const float2 lo = unpack2(q_lo), hi = unpack2(q_hi);
+      qd[lane] = pack2(lo.x * c0 - hi.x * s0, lo.y * c1 - hi.y * s1);
+      qd[lane + 32] = pack2(hi.x * c0 + lo.x * s0, hi.y * c1 + lo.y * s1);
     }
     {
-      const uint32_t* src = reinterpret_cast<const uint32_t*>(p.k_new + b * p.kn_sb + h * p.kn_sh + t * p.kn_st);
-      uint32_t* dst = reinterpret_cast<uint32_t*>(p.k_cache + b * p.kc_sb + h * p.kc_sh + slot * p.kc_ss);
-      const float2 lo = unpack2(src[lane]), hi = unpack2(src[lane + 32]);
-      dst[lane] = pack2(lo.x * c0 - hi.x * s0, lo.y * c1 - hi.y * s1);
-      dst[lane + 32] = pack2(hi.x * c0 + lo.x * s0, hi.y * c1 + lo.y * s1);
+      const float2 lo = unpack2(k_lo), hi = unpack2(k_hi);
+      kd[lane] = pack2(lo.x * c0 - hi.x * s0, lo.y * c1 - hi.y * s1);
+      kd[lane + 32] = pack2(hi.x * c0 + lo.x * s0, hi.y * c1 + lo.y * s1);
     }
-    {
-      const uint32_t* src = reinterpret_cast<const uint32_t*>(p.v_new + b * p.vn_sb + h * p.vn_sh + t * p.vn_st);
-      uint32_t* dst = reinterpret_cast<uint32_t*>(p.v_cache + b * p.vc_sb + h * p.vc_sh + slot * p.vc_ss);
-      dst[lane] = src[lane];
-      dst[lane + 32] = src[lane + 32];
-    }
+    vd[lane] = v_lo;
+    vd[lane + 32] = v_hi;
   }
 }
 
@@ -142,9 +146,10 @@ extern "C" int specvlm_rope_append(const uint16_t* q_in, const uint16_t* k_new, 
   p.vc_sb = d->vc_stride_b; p.vc_sh = d->vc_stride_h; p.vc_ss = d->vc_stride_s;
   const double base = d->rope_base > 0.f ? static_cast<double>(d->rope_base) : 10000.0;
   for (int i = 0; i < 64; ++i) p.inv_freq[i] = pow(base, -2.0 * i / 128.0);
-  // enough blocks along z that a warp handles one or two heads
-  int gz = (d->H + 2 * (kRopeThreads / 32) - 1) / (2 * (kRopeThreads / 32));
-  if (static_cast<int64_t>(gz) * d->T * d->B > 4096) gz = 1;
+  // one head per warp (every warp then makes a single memory round trip) while that keeps the grid
+  // moderate; larger batches loop over heads inside a warp
+  int gz = (d->H + (kRopeThreads / 32) - 1) / (kRopeThreads / 32);
+  while (gz > 1 && static_cast<int64_t>(gz) * d->T * d->B > 16384) gz = (gz + 1) / 2;
   dim3 grid(d->T, d->B, gz);
   return check_cuda(launch_overlapped(rope_append_kernel, grid, dim3(kRopeThreads), static_cast<cudaStream_t>(stream), p),
                     "rope_append launch");
