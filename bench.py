@@ -359,8 +359,9 @@ def run_ours(args, cfg):
     desc_pipe = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0], flags=sv.ATTN_FLAG_INPUTS_STABLE)
     # layer 0 of a pipelined step: the compaction kernel before it only writes tree slots, so the
     # prefix may be prefetched early; half-SM configuration so that layer 1 can overlap it
+    # (with a single layer there is no later launch to overlap: the whole-SM configuration is kept)
     desc_pipe0 = sv.make_attn_desc(q[0], k_cache[0], v_cache[0], out[0],
-                                   flags=sv.ATTN_FLAG_PREFIX_STABLE | sv.ATTN_FLAG_HALF_SM)
+                                   flags=sv.ATTN_FLAG_PREFIX_STABLE | (sv.ATTN_FLAG_HALF_SM if L > 1 else 0))
     ws = sv.alloc_attn_workspace(desc_ser, dev)
     launches_per_step = L + 3  # L attention launches, argmax, accept + compaction, tree_build
 
