@@ -74,6 +74,14 @@ def test_rope_append_matches_oracle(T):
     run_case(T, B=3, H=5, T=T, prefixes=[0, 333, 9728])
 
 
+@pytest.mark.parametrize("B,H", [(1, 32), (2, 40), (70, 9)])
+def test_rope_append_head_distribution_over_blocks(B, H):
+    """One head per warp (H a multiple of the warps per block or not), and a batch large enough
+    that a warp loops over several heads."""
+    rng = np.random.default_rng(B * H)
+    run_case(B * 100 + H, B=B, H=H, T=60, prefixes=rng.integers(0, 120, size=B).tolist())
+
+
 def test_rope_append_in_place_custom_base_and_strided_cache():
     run_case(99, B=2, H=4, T=60, prefixes=[3008, 17], base=500000.0, in_place=True)
 
