@@ -655,8 +655,12 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
   const bool aborted0 = *abort_flag != 0;
   if (threadIdx.x == 0) mbar_expect_tx(LAND_FULL, (ns - 1) * group_bytes);  // armed before anyone may send
   if (warp >= kSoftmaxWarp0 && !aborted0) {
-    float* d0 = stage + ((row0 % ns) * rk + row0 / ns) * kLandStride + t4 * 2;
-    float* d1 = stage + ((row1 % ns) * rk + row1 / ns) * kLandStride + t4 * 2;
+    // Within a row the 128 values are rotated by 8 columns per owner: the eight rows a warp stores
+    // at once then fall into different banks (rows of different owners are a multiple of 32 words
+    // apart otherwise). The owner undoes the rotation when it reads.
+    const int o0 = row0 % ns, o1 = row1 % ns;
+    float* d0 = stage + (o0 * rk + row0 / ns) * kLandStride;
+    float* d1 = stage + (o1 * rk + row1 / ns) * kLandStride;
     float ov[4][16];
     if (have_o) {
 #pragma unroll
@@ -672,8 +676,9 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
     for (int c = 0; c < 4; ++c) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        *reinterpret_cast<float2*>(d0 + c * 32 + j * 8) = make_float2(ov[c][4 * j + 0], ov[c][4 * j + 1]);
-        *reinterpret_cast<float2*>(d1 + c * 32 + j * 8) = make_float2(ov[c][4 * j + 2], ov[c][4 * j + 3]);
+        const int col = c * 32 + j * 8 + t4 * 2;
+        *reinterpret_cast<float2*>(d0 + ((col + 8 * o0) & (kD - 1))) = make_float2(ov[c][4 * j + 0], ov[c][4 * j + 1]);
+        *reinterpret_cast<float2*>(d1 + ((col + 8 * o1) & (kD - 1))) = make_float2(ov[c][4 * j + 2], ov[c][4 * j + 3]);
       }
     }
     if (t4 == 0) {
@@ -710,26 +715,31 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
     for (int k = sw + 4 * rr; k < rk; k += 16) {
       const int row = split + k * ns;
       if (row < T) {
+        // all sources' (max, sum) pairs first, then all value loads: nothing here depends on a
+        // previous shared-memory load (at most 8 splits reach this path)
+        const float* srcs[8];
+        float2 ml[8];
         float mstar = -INFINITY;
-#pragma unroll 1
-        for (int s2 = 0; s2 < ns; ++s2) {
-          const float* src = (s2 == split ? stage + split * rk * kLandStride : landp + s2 * rk * kLandStride) + k * kLandStride;
-          mstar = fmaxf(mstar, src[kD]);
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) {
+          srcs[s2] = (s2 == split ? stage + split * rk * kLandStride : landp + s2 * rk * kLandStride) + k * kLandStride;
+          ml[s2] = s2 < ns ? *reinterpret_cast<const float2*>(srcs[s2] + kD) : make_float2(-INFINITY, 0.f);
+          mstar = fmaxf(mstar, ml[s2].x);
         }
         float4 acc[4];
 #pragma unroll
         for (int q4 = 0; q4 < 4; ++q4) acc[q4] = make_float4(0.f, 0.f, 0.f, 0.f);
         float lsum = 0.f;
-#pragma unroll 1
-        for (int s2 = 0; s2 < ns; ++s2) {
-          const float* src = (s2 == split ? stage + split * rk * kLandStride : landp + s2 * rk * kLandStride) + k * kLandStride;
-          const float2 ml = *reinterpret_cast<const float2*>(src + kD);
-          const float w = (ml.x == -INFINITY) ? 0.f : ex2(ml.x - mstar);
-          lsum += w * ml.y;
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const float4 x = *(reinterpret_cast<const float4*>(src + cc * 16) + q4);
-            acc[q4].x += w * x.x; acc[q4].y += w * x.y; acc[q4].z += w * x.z; acc[q4].w += w * x.w;
+        for (int s2 = 0; s2 < 8; ++s2) {
+          if (s2 < ns) {
+            const float w = (ml[s2].x == -INFINITY) ? 0.f : ex2(ml[s2].x - mstar);
+            lsum += w * ml[s2].y;
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              const float4 x = *reinterpret_cast<const float4*>(srcs[s2] + ((cc * 16 + q4 * 4 + 8 * split) & (kD - 1)));
+              acc[q4].x += w * x.x; acc[q4].y += w * x.y; acc[q4].z += w * x.z; acc[q4].w += w * x.w;
+            }
           }
         }
         const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
