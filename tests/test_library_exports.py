@@ -62,3 +62,53 @@ def test_host_side_argument_errors_need_no_gpu():
     # null pointers are rejected before any launch
     assert lib.specvlm_argmax(None, 1, 60, 32000, 32000, None, None) == -1
     assert lib.specvlm_tree_build(None, None, 1, 60, None, None, None, None, None) == -1
+
+
+def _header_prototypes():
+    """name -> list of parameter kinds ('ptr', 'i32', 'i64', 'f32', 'size') parsed from the header."""
+    text = open(os.path.join(ROOT, "include", "specvlm.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    protos = {}
+    for name, args in re.findall(r"SPECVLM_API[^;(]*?\b(specvlm_\w+)\s*\(([^)]*)\)\s*;", text):
+        kinds = []
+        args = " ".join(args.split())
+        if args not in ("", "void"):
+            for a in args.split(","):
+                a = a.strip()
+                if "*" in a:
+                    kinds.append("ptr")
+                elif re.match(r"(const\s+)?int64_t\b", a):
+                    kinds.append("i64")
+                elif re.match(r"(const\s+)?(int32_t|int)\b", a):
+                    kinds.append("i32")
+                elif re.match(r"(const\s+)?float\b", a):
+                    kinds.append("f32")
+                elif re.match(r"(const\s+)?size_t\b", a):
+                    kinds.append("size")
+                else:
+                    raise AssertionError(f"unparsed parameter {a!r} of {name}")
+        protos[name] = kinds
+    return protos
+
+
+def test_binding_prototypes_match_the_header():
+    """Every ctypes prototype has the header's parameter count, and pointers / 32-bit / 64-bit /
+    float parameters sit where the header puts them (a mismatch would corrupt the call silently)."""
+    import ctypes
+    lib = sv.load_library()
+    kinds_of = {ctypes.c_int32: "i32", ctypes.c_int: "i32", ctypes.c_int64: "i64", ctypes.c_float: "f32",
+                ctypes.c_size_t: "size", ctypes.c_void_p: "ptr", ctypes.c_char_p: "ptr"}
+    protos = _header_prototypes()
+    assert sorted(protos) == _declared()
+    for name, want in protos.items():
+        argtypes = getattr(lib, name).argtypes
+        assert argtypes is not None, f"{name} has no ctypes prototype"
+        got = []
+        for t in argtypes:
+            if t in kinds_of:
+                got.append(kinds_of[t])
+            elif hasattr(t, "contents") or getattr(t, "_type_", None) is not None and not isinstance(t._type_, str):
+                got.append("ptr")          # POINTER(struct)
+            else:
+                raise AssertionError(f"unknown ctypes type {t} in {name}")
+        assert got == want, f"{name}: binding {got} != header {want}"
