@@ -70,3 +70,41 @@ def test_mask_written_by_tree_build_is_seen_by_overlapping_attention_launches():
         got = out.float().cpu().numpy()[:, 0, :, :, :]          # [L][H][T][D]
         err = np.abs(got - want[which][None, None, :, None]).max(axis=(1, 2, 3))
         assert err.max() < 4e-3, (trial, which, err)
+
+
+def test_back_to_back_launches_of_mixed_shapes_and_flags():
+    """Launches of different shapes, split counts and overlap flags enqueued without a host
+    synchronisation in between (each on its own tensors, so every promise the flags make holds):
+    whole-SM and half-SM configurations follow one another and overlap; every output must still
+    match the oracle."""
+    import sys
+    import os
+    sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+    from util import assert_attn_close, bits_to_torch, mask_to_torch, oracle_attn_all, torch_to_bits
+    rng = np.random.default_rng(2024)
+    cases = []
+    for c in range(18):
+        B, H, T = int(rng.integers(1, 4)), int(rng.integers(1, 40)), int(rng.integers(1, 65))
+        prefixes = [int(x) for x in rng.integers(0, int(rng.choice([100, 700, 3000])), size=B)]
+        S_cap = max(prefixes) + T + int(rng.integers(0, 70))
+        parents = [wl.eagle2_like_tree(rng, T, min(6, T - 1)) if T >= 20 else
+                   (wl.config1_tree(rng, T, min(4, T - 1)) if T > 1 else wl.single_node_tree()) for _ in range(B)]
+        masks = np.array([oracle.tree_mask_bits(p) for p in parents])
+        q = wl.normal_bf16_bits(rng, (B, H, T, 128))
+        k = wl.normal_bf16_bits(rng, (B, H, S_cap, 128))
+        v = wl.normal_bf16_bits(rng, (B, H, S_cap, 128))
+        flags = int(rng.choice([0, sv.ATTN_FLAG_PREFIX_STABLE, sv.ATTN_FLAG_INPUTS_STABLE, sv.ATTN_FLAG_INPUTS_STABLE,
+                                sv.ATTN_FLAG_PREFIX_STABLE | sv.ATTN_FLAG_HALF_SM]))
+        splits = int(rng.choice([0, 0, 1, 2, 4, 8]))
+        tq, tk, tv = bits_to_torch(q), bits_to_torch(k), bits_to_torch(v)
+        cases.append((q, k, v, prefixes, masks, tq, tk, tv, torch.full_like(tq, 7.0),
+                      torch.tensor(prefixes, dtype=torch.int32, device="cuda"), mask_to_torch(masks), flags, splits))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    for (_, _, _, _, _, tq, tk, tv, out, tpl, tm, flags, splits) in cases:
+        desc = sv.make_attn_desc(tq, tk, tv, out, splits, 0.0, flags)
+        sv.specvlm_tree_verify_attn(tq, tk, tv, tpl, None, tm, out, status=status, desc=desc)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    for (q, k, v, prefixes, masks, _, _, _, out, _, _, _, _) in cases:
+        assert_attn_close(torch_to_bits(out), oracle_attn_all(q, k, v, prefixes, masks))
