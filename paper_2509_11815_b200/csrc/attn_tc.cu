@@ -105,6 +105,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// Non-blocking poll. mbarrier.try_wait may suspend the thread for a system-dependent time when the
+// phase is not complete; the producer and the MMA issuer poll several barriers in turn and must
+// not sleep on one while another is ready, so they use test_wait.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait: false after kSpinLimit unsuccessful polls or once another role has given up.
 __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
@@ -343,11 +353,11 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
       uint32_t idle = 0;
       while (ik < n_tiles || iv < n_tiles) {
         bool progress = false;
-        if (ik < n_tiles && (ik < kKStages || mbar_try_wait(EMPTY_K(ik % kKStages), ((ik / kKStages) & 1) ^ 1))) {
+        if (ik < n_tiles && (ik < kKStages || mbar_test(EMPTY_K(ik % kKStages), ((ik / kKStages) & 1) ^ 1))) {
           issue_k(ik++);
           progress = true;
         }
-        if (iv < n_tiles && (iv < kVStages || mbar_try_wait(EMPTY_V(iv % kVStages), ((iv / kVStages) & 1) ^ 1))) {
+        if (iv < n_tiles && (iv < kVStages || mbar_test(EMPTY_V(iv % kVStages), ((iv / kVStages) & 1) ^ 1))) {
           issue_v(iv++);
           progress = true;
         }
@@ -419,13 +429,13 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
       uint32_t idle = 0;
       while (ok && ip < n_tiles) {
         bool progress = false;
-        if (ip < iq && mbar_try_wait(P_FULL, ip & 1) && mbar_try_wait(FULL_V(v_stage), v_parity)) {
+        if (ip < iq && mbar_test(P_FULL, ip & 1) && mbar_test(FULL_V(v_stage), v_parity)) {
           tc_fence_after();
           issue_pv(ip++);
           progress = true;
         }
-        if (iq < n_tiles && iq < ip + 2 && mbar_try_wait(FULL_K(k_stage), k_parity) &&
-            (iq < 2 || mbar_try_wait(S_FREE(iq & 1), ((iq >> 1) & 1) ^ 1))) {
+        if (iq < n_tiles && iq < ip + 2 && mbar_test(FULL_K(k_stage), k_parity) &&
+            (iq < 2 || mbar_test(S_FREE(iq & 1), ((iq >> 1) & 1) ^ 1))) {
           tc_fence_after();
           issue_qk(iq++);
           progress = true;
