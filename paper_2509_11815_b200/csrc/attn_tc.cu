@@ -41,7 +41,8 @@ constexpr int kD = SPECVLM_HEAD_DIM;
 constexpr int kRows = 64;      // MMA M: padded tree queries
 constexpr int kThreads = 192;
 constexpr int kSoftmaxWarp0 = 2;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 22;      // polls of a possibly suspending try_wait
+constexpr uint32_t kPollLimit = 1u << 25;      // turns of a non-blocking polling loop (well under a second)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units; P stays <= 2^8
 constexpr int kLandStride = kD + 4;        // floats per exchange row: 128 values, (max, sum), padding
 
@@ -363,7 +364,7 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
         }
         if (progress) {
           idle = 0;
-        } else if (++idle > kSpinLimit || ((idle & 1023u) == 0 && *abort_flag)) {
+        } else if (++idle > kPollLimit || ((idle & 1023u) == 0 && *abort_flag)) {
           *abort_flag = 1;
           break;
         }
@@ -442,7 +443,7 @@ tree_attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap map_
         }
         if (progress) {
           idle = 0;
-        } else if (++idle > kSpinLimit || ((idle & 1023u) == 0 && *abort_flag)) {
+        } else if (++idle > kPollLimit || ((idle & 1023u) == 0 && *abort_flag)) {
           *abort_flag = 1;
           ok = false;
         }
